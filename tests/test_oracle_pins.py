@@ -1,0 +1,329 @@
+"""Pins for the CPU oracle: hand-worked fixtures, closed forms, invariants, library routines
+and brute force. None of these tests touches the CUDA library."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ec_oracle as orc
+from paper_2407_18121_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    with open(os.path.join(GOLDEN, name)) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def _bf16(x):
+    return wl.to_bf16_bits(np.asarray(x, np.float32))
+
+
+def _rand_bits(rng, shape, sigma=1.0):
+    return _bf16(rng.standard_normal(shape).astype(np.float32) * sigma)
+
+
+# ------------------------------------------------------------------ importance (Eq. 1)
+
+def test_importance_hand_example():
+    rows = _rows("importance_pow2.txt")
+    q = _bf16(np.ones((1, 3, 1)))
+    k = _bf16(np.array([0.0, 1.0, 2.0]).reshape(1, 3, 1))
+    scores, lse = orc.importance(q, k, math.log(2.0))
+    want = np.array([float(Fraction(int(a), int(b))) for a, b, _ in rows])
+    want_lse = np.array([math.log(float(c)) for _, _, c in rows])
+    np.testing.assert_allclose(scores[0], want, rtol=1e-14)
+    np.testing.assert_allclose(lse[0], want_lse, rtol=0, atol=1e-14)
+
+
+def test_importance_zero_queries_is_harmonic():
+    # uniform attention: I_n = sum_{m>=n} 1/(m+1) = H_T - H_n
+    T, D = 37, 8
+    rng = np.random.default_rng(0)
+    q = _bf16(np.zeros((2, T, D)))
+    k = _rand_bits(rng, (2, T, D))
+    scores, lse = orc.importance(q, k, 0.7)
+    want = np.array([sum(1.0 / (m + 1) for m in range(n, T)) for n in range(T)])
+    np.testing.assert_allclose(scores[0], want, rtol=1e-13)
+    np.testing.assert_allclose(scores[1], want, rtol=1e-13)
+    np.testing.assert_allclose(lse[0], np.log(np.arange(1, T + 1)), atol=1e-13)
+
+
+@pytest.mark.parametrize("T,D,scale", [(1, 4, 1.0), (2, 4, 0.3), (16, 8, 1.0), (45, 16, 0.25)])
+def test_importance_matches_library_softmax(T, D, scale):
+    rng = np.random.default_rng(T * 100 + D)
+    qb, kb = _rand_bits(rng, (3, T, D)), _rand_bits(rng, (3, T, D))
+    scores, lse = orc.importance(qb, kb, scale)
+    q = torch.from_numpy(wl.bf16_bits_to_f64(qb))
+    k = torch.from_numpy(wl.bf16_bits_to_f64(kb))
+    logits = scale * q @ k.transpose(-1, -2)
+    mask = torch.tril(torch.ones(T, T, dtype=torch.bool))
+    logits = logits.masked_fill(~mask, float("-inf"))
+    A = torch.softmax(logits, dim=-1)
+    np.testing.assert_allclose(scores, A.sum(dim=-2).numpy(), rtol=1e-12)
+    np.testing.assert_allclose(lse, torch.logsumexp(logits, dim=-1).numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_importance_operands_not_transposed():
+    # asymmetric case: only the q.k order that puts QUERIES on rows gives this answer
+    T, D = 5, 3
+    rng = np.random.default_rng(5)
+    qb, kb = _rand_bits(rng, (1, T, D), 2.0), _rand_bits(rng, (1, T, D), 2.0)
+    s_qk, _ = orc.importance(qb, kb, 1.0)
+    s_kq, _ = orc.importance(kb, qb, 1.0)
+    assert np.abs(s_qk - s_kq).max() > 1e-3
+    q, k = wl.bf16_bits_to_f64(qb)[0], wl.bf16_bits_to_f64(kb)[0]
+    I = np.zeros(T)
+    for m in range(T):
+        w = np.array([math.exp(float(q[m] @ k[n])) for n in range(m + 1)])
+        I[: m + 1] += w / w.sum()
+    np.testing.assert_allclose(s_qk[0], I, rtol=1e-12)
+
+
+def test_importance_invariants():
+    T, D = 64, 16
+    rng = np.random.default_rng(7)
+    qb, kb = _rand_bits(rng, (4, T, D)), _rand_bits(rng, (4, T, D))
+    scores, _ = orc.importance(qb, kb, 0.5)
+    np.testing.assert_allclose(scores.sum(-1), T, rtol=1e-12)   # rows of A sum to one
+    assert (scores[:, 0] >= 1.0).all()                           # A[0][0] = 1
+    assert (scores[:, -1] <= 1.0).all() and (scores > 0).all()
+
+
+def test_layer_mean():
+    rng = np.random.default_rng(1)
+    s = rng.random((3, 5, 11))
+    np.testing.assert_allclose(orc.layer_mean(s), s.mean(axis=1), rtol=1e-14)
+
+
+# ------------------------------------------------------------------ keep count / selection
+
+def test_keep_counts_of_the_five_configurations():
+    got = []
+    for name in wl.CONFIG_ORDER:
+        w = wl.WORKLOADS[name]
+        got.append([orc.keep_count(w.prompt_len, r) for r in w.keep_ratios])
+    assert got == [[128], [320], [256], [205, 512, 1024, 1536], [820]]
+    assert orc.keep_count(100, 1.0) == 100 and orc.keep_count(100, 0.0) == 1
+
+
+def _brute_select(s, C, protect):
+    s = np.array(s, np.float64)
+    T = len(s)
+    if protect:
+        s[0] = np.inf
+        if C >= 2:
+            s[-1] = np.inf
+    order = sorted(range(T), key=lambda i: (-s[i], i))
+    return np.array(sorted(order[:C]), np.int32)
+
+
+@pytest.mark.parametrize("protect", [False, True])
+def test_select_brute_force_with_ties(protect):
+    rng = np.random.default_rng(3)
+    for T, C in [(1, 1), (2, 1), (2, 2), (9, 1), (9, 4), (33, 33), (40, 17)]:
+        s = rng.integers(0, 6, size=(5, T)).astype(np.float64)   # many exact ties
+        got = orc.select(s, C, protect)
+        for u in range(5):
+            np.testing.assert_array_equal(got[u], _brute_select(s[u], C, protect))
+
+
+def test_select_known_top_set_and_order():
+    s = np.array([[0.1, 5.0, 0.2, 4.0, 0.3, 3.0, 0.0]])
+    np.testing.assert_array_equal(orc.select(s, 3, False)[0], [1, 3, 5])
+    np.testing.assert_array_equal(orc.select(s, 3, True)[0], [0, 1, 6])
+    np.testing.assert_array_equal(orc.select(s, 7, False)[0], np.arange(7))
+    # lower position wins a tie
+    t = np.array([[1.0, 2.0, 2.0, 2.0]])
+    np.testing.assert_array_equal(orc.select(t, 2, False)[0], [1, 2])
+
+
+def test_select_threshold_property():
+    rng = np.random.default_rng(11)
+    s = rng.random((6, 200))
+    a = orc.select(s, 50, False)
+    for u in range(6):
+        assert (np.diff(a[u]) > 0).all() and len(a[u]) == 50
+        rest = np.setdiff1d(np.arange(200), a[u])
+        assert s[u, a[u]].min() >= s[u, rest].max()
+
+
+# ------------------------------------------------------------------ buckets (Eq. 2), merge (Eq. 3)
+
+def test_bucket_merge_hand_example():
+    rows = _rows("bucket_merge_example.txt")
+    T, D = 7, 2
+    X = np.array([[t, 10 - 2 * t] for t in range(T)], np.float32).reshape(1, T, D)
+    anchors = np.array([[0, 3, 4]], np.int32)
+    lo, hi = orc.buckets(anchors, T)
+    assert lo[0].tolist() == [int(r[0]) for r in rows]
+    assert hi[0].tolist() == [int(r[1]) for r in rows]
+    m = orc.merge(_bf16(X), lo, hi)
+    want = np.array([[float(r[2]), float(r[3])] for r in rows])
+    np.testing.assert_allclose(m[0], want, rtol=1e-15)
+
+
+def test_buckets_are_nearest_anchor_ties_to_earlier():
+    rng = np.random.default_rng(2)
+    for T, C in [(1, 1), (5, 1), (8, 8), (30, 7), (64, 20), (65, 2)]:
+        a = np.sort(rng.choice(T, size=C, replace=False)).astype(np.int32)[None]
+        lo, hi = orc.buckets(a, T)
+        owner = np.full(T, -1)
+        for k in range(C):
+            assert lo[0, k] <= a[0, k] <= hi[0, k]
+            assert (owner[lo[0, k]: hi[0, k] + 1] == -1).all()
+            owner[lo[0, k]: hi[0, k] + 1] = k
+        assert (owner >= 0).all()
+        for t in range(T):
+            d = np.abs(a[0].astype(np.int64) - t)
+            assert owner[t] == int(np.argmin(d))     # argmin returns the first = earlier anchor
+
+
+def test_merge_properties():
+    rng = np.random.default_rng(4)
+    U, T, D, C = 3, 50, 8, 9
+    Xb = _rand_bits(rng, (U, T, D))
+    X = wl.bf16_bits_to_f64(Xb)
+    anchors = np.stack([np.sort(rng.choice(T, C, replace=False)) for _ in range(U)]).astype(np.int32)
+    lo, hi = orc.buckets(anchors, T)
+    m = orc.merge(Xb, lo, hi)
+    size = (hi - lo + 1).astype(np.float64)
+    np.testing.assert_allclose((m * size[..., None]).sum(1), X.sum(1), rtol=1e-12, atol=1e-12)
+    # explicit per-bucket numpy mean
+    for u in range(U):
+        for k in range(C):
+            np.testing.assert_allclose(m[u, k], X[u, lo[u, k]: hi[u, k] + 1].mean(0), rtol=1e-13, atol=1e-15)
+    # one anchor: global mean; all anchors: identity, bit for bit after rounding back
+    one = np.array([[17]] * U, np.int32)
+    l1, h1 = orc.buckets(one, T)
+    np.testing.assert_allclose(orc.merge(Xb, l1, h1)[:, 0], X.mean(1), rtol=1e-13)
+    full = np.tile(np.arange(T, dtype=np.int32), (U, 1))
+    lf, hf = orc.buckets(full, T)
+    np.testing.assert_array_equal(orc.round_bf16(orc.merge(Xb, lf, hf)), Xb)
+    # constant rows stay constant
+    const = _bf16(np.full((1, 20, 4), 1.5))
+    lc, hc = orc.buckets(np.array([[3, 9, 15]], np.int32), 20)
+    assert (orc.merge(const, lc, hc) == 1.5).all()
+
+
+def test_round_bf16_is_round_to_nearest_even():
+    # 1 + 2^-8 is the midpoint between bf16 neighbours 1 and 1 + 2^-7: tie goes to even (1.0)
+    x = np.array([1.0 + 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -30, 1.0 + 3 * 2.0 ** -8, -2.5, 0.0, 1e-3])
+    got = wl.bf16_bits_to_f64(orc.round_bf16(x))
+    assert got[0] == 1.0 and got[1] == 1.0 + 2.0 ** -7 and got[2] == 1.0 + 2.0 ** -6 and got[3] == -2.5
+    assert got[4] == 0.0 and abs(got[5] - 1e-3) <= 1e-3 * 2.0 ** -8
+    # agrees with torch's float32 -> bfloat16 on float32-representable values
+    rng = np.random.default_rng(0)
+    f = rng.standard_normal(4096).astype(np.float32)
+    tb = torch.from_numpy(f).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(orc.round_bf16(f.astype(np.float64)), tb)
+    np.testing.assert_array_equal(wl.to_bf16_bits(f), tb)
+    np.testing.assert_array_equal(orc.widen_bf16(tb), torch.from_numpy(tb.view(np.int16)).view(torch.bfloat16).double().numpy())
+
+
+# ------------------------------------------------------------------ decode attention + eviction
+
+def test_decode_hand_example():
+    want = float(_rows("decode_pow2.txt")[0][0])
+    K0 = np.array([[0.0], [1.0]]).reshape(1, 2, 1)
+    V0 = np.array([[1.0], [2.0]]).reshape(1, 2, 1)
+    qd = orc.DecodeQueue(K0, V0, cap=4)
+    out, pos, ident = qd.step(_bf16([[1.0]]), _bf16([[2.0]]), _bf16([[4.0]]), math.log(2.0),
+                              policy=orc.POLICY_FIXED, budget=8, offset=1)
+    assert abs(out[0, 0] - want) < 1e-14 and pos == -1 and ident == -1 and qd.len == 3
+
+
+def test_decode_matches_library_softmax_and_special_cases():
+    rng = np.random.default_rng(9)
+    U, L, D = 4, 23, 16
+    K0 = wl.bf16_bits_to_f64(_rand_bits(rng, (U, L, D)))
+    V0 = wl.bf16_bits_to_f64(_rand_bits(rng, (U, L, D)))
+    qb, kb, vb = _rand_bits(rng, (U, D)), _rand_bits(rng, (U, D)), _rand_bits(rng, (U, D))
+    qd = orc.DecodeQueue(K0, V0, cap=L + 1)
+    out, _, _ = qd.step(qb, kb, vb, 0.25, policy=orc.POLICY_FIXED, budget=L + 1, offset=3)
+    Kall = torch.from_numpy(np.concatenate([K0, wl.bf16_bits_to_f64(kb)[:, None]], 1))
+    Vall = torch.from_numpy(np.concatenate([V0, wl.bf16_bits_to_f64(vb)[:, None]], 1))
+    q = torch.from_numpy(wl.bf16_bits_to_f64(qb))
+    p = torch.softmax(0.25 * torch.einsum("ud,uld->ul", q, Kall), dim=-1)
+    want = torch.einsum("ul,uld->ud", p, Vall).numpy()
+    np.testing.assert_allclose(out, want, rtol=1e-12, atol=1e-14)
+    # convex combination
+    assert (out <= Vall.numpy().max(1) + 1e-12).all() and (out >= Vall.numpy().min(1) - 1e-12).all()
+    # q = 0 -> plain mean of all value rows (cache and new)
+    qd0 = orc.DecodeQueue(K0, V0, cap=L + 1)
+    out0, _, _ = qd0.step(_bf16(np.zeros((U, D))), kb, vb, 0.25, policy=0, budget=L + 1, offset=3)
+    np.testing.assert_allclose(out0, Vall.numpy().mean(1), rtol=1e-13, atol=1e-15)
+    # permuting cached rows leaves the output unchanged
+    perm = rng.permutation(L)
+    qdp = orc.DecodeQueue(K0[:, perm], V0[:, perm], cap=L + 1)
+    outp, _, _ = qdp.step(qb, kb, vb, 0.25, policy=0, budget=L + 1, offset=3)
+    np.testing.assert_allclose(outp, out, rtol=1e-12, atol=1e-14)
+
+
+def test_fixed_point_queue_hand_example():
+    rows = _rows("fixed_point_queue.txt")
+    rng = np.random.default_rng(0)
+    K0 = rng.standard_normal((2, 5, 4))
+    qd = orc.DecodeQueue(K0, K0.copy(), cap=6)
+    for r in rows:
+        kb = _rand_bits(rng, (2, 4))
+        _, pos, ident = qd.step(kb, kb, kb, 1.0, policy=orc.POLICY_FIXED, budget=5, offset=2)
+        assert pos == int(r[1]) and ident == int(r[2])
+        assert qd.identities().tolist() == [int(x) for x in r[3:]]
+
+
+def test_fixed_point_retained_set_and_contents():
+    rng = np.random.default_rng(12)
+    C, d, D, steps = 12, 4, 4, 19
+    K0 = wl.bf16_bits_to_f64(_rand_bits(rng, (1, C, D)))
+    qd = orc.DecodeQueue(K0, K0.copy(), cap=C + 1)
+    newk = []
+    for s in range(steps):
+        kb = _rand_bits(rng, (1, D))
+        newk.append(wl.bf16_bits_to_f64(kb)[0])
+        _, pos, ident = qd.step(kb, kb, kb, 1.0, policy=0, budget=C, offset=d)
+        assert qd.len == C and pos == C - d                      # fixed truncation location
+        ids = qd.identities()
+        recent = list(range(C + s - d + 1, C + s + 1))
+        assert ids.tolist() == list(range(C - d)) + recent       # first C-d rows + d newest
+        assert ident == (C - d + s)                              # rows leave in arrival order
+        for j, i in enumerate(ids):                              # rows moved with their identities
+            src = K0[0, i] if i < C else newk[i - C]
+            np.testing.assert_array_equal(qd.K[0, j], src)
+
+
+def test_below_budget_nothing_is_evicted():
+    rng = np.random.default_rng(13)
+    K0 = rng.standard_normal((1, 3, 4))
+    qd = orc.DecodeQueue(K0, K0.copy(), cap=8)
+    for s in range(4):
+        kb = _rand_bits(rng, (1, 4))
+        _, pos, _ = qd.step(kb, kb, kb, 1.0, policy=0, budget=6, offset=2)
+        assert pos == (-1 if s < 3 else 4)
+    assert qd.len == 6
+
+
+def test_ratio_policy_follows_algorithm_1_count():
+    # direct simulation of del_num = int(seq_len - n * ratio): one row leaves whenever it reaches 1
+    rng = np.random.default_rng(14)
+    T, ratio, d = 40, 0.3, 5
+    C = orc.keep_count(T, ratio)
+    K0 = rng.standard_normal((1, C, 4))
+    qd = orc.DecodeQueue(K0, K0.copy(), cap=C + 40)
+    length = C
+    for s in range(30):
+        n_tot = T + s + 1
+        kb = _rand_bits(rng, (1, 4))
+        _, pos, _ = qd.step(kb, kb, kb, 1.0, policy=orc.POLICY_RATIO, offset=d, ratio=ratio, n_tot=n_tot)
+        length += 1
+        if int(length - n_tot * ratio) >= 1:
+            assert pos == length - 1 - d
+            length -= 1
+        else:
+            assert pos == -1
+        assert qd.len == length
+        assert length <= n_tot * ratio + 1
