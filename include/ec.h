@@ -1,0 +1,185 @@
+/*
+ * ec.h — C ABI of the Elastic Cache hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the cache manager of "Efficient Inference of Vision
+ * Instruction-Following Models with Elastic Cache" (arXiv 2407.18121), Sec. 3.3 and
+ * Algorithm 1, as CUDA kernels:
+ *
+ *   ec_importance    per-head importance of every prompt key (Eq. 1 + column sums)
+ *   ec_select_merge  anchor selection, bucket division (Eq. 2) and mean merge (Eq. 3)
+ *                    into a dense compacted cache with an index map
+ *   ec_decode_step   single-query attention over the compacted cache plus the new token,
+ *                    followed by fixed-point elimination (in-place slot reuse)
+ *
+ * Conventions shared by every call
+ *  - Pointers named "dev" are CUDA device pointers of the current device; "host" pointers
+ *    are ordinary host memory. The caller owns every buffer. The library allocates no
+ *    device memory and keeps no state between calls.
+ *  - bf16 tensors are passed as `const void*` to 2-byte elements, row-major, innermost
+ *    dimension contiguous, base address 16-byte aligned. D (head_dim) is 64 or 128.
+ *  - N counts independent problems (batch x layers folded), H heads per problem. A "unit"
+ *    is one (problem, head) pair; units never interact except through EC_LAYER_SHARED.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream). Calls only enqueue
+ *    work; they return after launch. Errors detectable on the host are returned at once and
+ *    nothing is launched; in that case outputs are untouched.
+ *  - Every function returns an ec_status as int. No function throws, aborts or prints.
+ *  - Workspace: each call states its scratch need through the matching *_workspace query;
+ *    the caller passes a device buffer of at least that many bytes, 256-byte aligned. The
+ *    first 256 bytes of an importance workspace hold a device status word (see
+ *    ec_device_status).
+ */
+#ifndef EC_H_
+#define EC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EC_OK = 0,
+    EC_ERR_NULL = 1,      /* a required pointer is NULL                                  */
+    EC_ERR_SHAPE = 2,     /* a dimension is out of the supported range                   */
+    EC_ERR_ALIGN = 3,     /* a pointer is not 16-byte (workspace: 256-byte) aligned      */
+    EC_ERR_ARG = 4,       /* a scalar argument is out of range                           */
+    EC_ERR_WORKSPACE = 5, /* workspace missing or smaller than the query reports         */
+    EC_ERR_CUDA = 6,      /* a CUDA runtime call failed (launch error, no device, ...)   */
+    EC_ERR_TIMEOUT = 7    /* a bounded device-side wait expired (see ec_device_status)   */
+} ec_status;
+
+/* Static description of a status code; never NULL. */
+const char *ec_status_string(int status);
+
+/*
+ * Number of anchors kept for a prompt of T tokens at retention ratio `keep_ratio`
+ * (gamma of Sec. 3.3). Follows Algorithm 1's count of removed entries at the prompt call,
+ * del = int(T - T*gamma), so the result is T - del, clamped to [1, T]. Host arithmetic in
+ * double. Returns 0 when T < 1 or the ratio is not in [0, 1].
+ */
+int ec_keep_count(int T, double keep_ratio);
+
+/* ---------------------------------------------------------------- importance ------- */
+
+/* Bytes of device scratch ec_importance needs for these shapes (0 on invalid shapes). */
+size_t ec_importance_workspace(int N, int H, int T, int D);
+
+/*
+ * Importance of every prompt key (Sec. 3.3, Eq. 1 and the definition that follows it):
+ *   A[m][n] = exp(scale*<q_m,k_n>) / sum_{n'<=m} exp(scale*<q_m,k_n'>)   for n <= m, else 0
+ *   scores[n] = sum_m A[m][n]
+ * per unit. The T x T matrix is never stored: a first pass computes each query row's
+ * log-sum-exp, a second pass accumulates the column sums.
+ *
+ *   Q_dev, K_dev   bf16 [N, H, T, D]                           (in)
+ *   scores_dev     fp32 [N, H, T]                              (out)
+ *   lse_dev        fp32 [N, H, T], natural log; may be NULL    (out, optional)
+ *   scale          multiplies the dot product (the paper's Eq. 1 has none: pass 1.0 with
+ *                  pre-scaled keys, or 1/sqrt(D) for a standard attention head)
+ *   ws_dev         scratch of ec_importance_workspace bytes
+ * Limits: 1 <= T <= 16384, N*H*T < 2^31, N*H < 2^24. Returns EC_OK or a host-detected error.
+ */
+int ec_importance(const void *Q_dev, const void *K_dev, float *scores_dev, float *lse_dev,
+                  int N, int H, int T, int D, float scale,
+                  void *ws_dev, size_t ws_bytes, void *stream);
+
+/*
+ * Synchronises `stream` and reports what the kernels recorded in the workspace's status
+ * word: EC_OK, or EC_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are
+ * then undefined but no out-of-bounds access happened). EC_ERR_CUDA on a runtime error.
+ */
+int ec_device_status(void *ws_dev, void *stream);
+
+/* ---------------------------------------------------------------- select + merge ---- */
+
+typedef enum {
+    EC_PER_HEAD = 0,     /* every head ranks its own scores                              */
+    EC_LAYER_SHARED = 1  /* scores are averaged over the heads of a problem first (the
+                            paper's layer-wise population); all heads share the anchors  */
+} ec_population;
+
+size_t ec_select_merge_workspace(int N, int H, int T, int D, int n_keep, int population);
+
+/*
+ * Anchor selection, bucket division and merging (Sec. 3.3; Eq. 2; Eq. 3).
+ *  1. anchors = the n_keep positions with the largest score (equal scores: the lower
+ *     position wins), listed ascending. With protect_ends != 0, position 0 and (when
+ *     n_keep >= 2) position T-1 are always anchors (Sec. 4.1, implementation details).
+ *  2. bucket k = positions floor((t_{k-1}+t_k)/2)+1 .. floor((t_k+t_{k+1})/2), the first
+ *     bucket starting at 0 and the last ending at T-1.
+ *  3. row k of the compacted cache = arithmetic mean of the bucket's rows (fp32
+ *     accumulation in position order, one rounding to bf16), for K and for V.
+ *
+ *   K_dev, V_dev    bf16 [N, H, T, D]                                     (in)
+ *   scores_dev      fp32 [N, H, T]                                        (in)
+ *   n_keep          1..T (see ec_keep_count)
+ *   Kc_dev, Vc_dev  bf16 [N, H, cap, D], rows 0..n_keep-1 written         (out), cap >= n_keep
+ *   anchor_pos_dev  int32 [N, H, n_keep], ascending prompt positions      (out) = index map
+ *   bucket_len_dev  int32 [N, H, n_keep], bucket sizes; may be NULL       (out, optional)
+ * The inputs must not overlap the outputs.
+ */
+int ec_select_merge(const void *K_dev, const void *V_dev, const float *scores_dev,
+                    int N, int H, int T, int D, int n_keep, int population, int protect_ends,
+                    void *Kc_dev, void *Vc_dev, int cap,
+                    int32_t *anchor_pos_dev, int32_t *bucket_len_dev,
+                    void *ws_dev, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------- decode ------------ */
+
+/*
+ * Host-side description of a compacted cache. Plain data: copy it to checkpoint it.
+ * Rows live in device buffers Kc, Vc of shape bf16 [N, H, cap, D]; `len` rows are valid.
+ * Because attention does not depend on row order, eviction does not shift rows: the new
+ * row is written into the physical slot of the evicted one. Slots [budget-offset, budget)
+ * form a ring that holds the `offset` most recent rows once the cache is full.
+ */
+typedef struct {
+    void *Kc, *Vc;      /* device, bf16 [N, H, cap, D]                                   */
+    int N, H, D, cap;
+    int len;            /* valid rows per unit (same for all units)                      */
+    int budget;         /* fixed-budget policy: rows kept after every step               */
+    int offset;         /* rows that stay behind the truncation location (>= 1)          */
+    int ring_head;      /* next ring slot to be reused, 0..offset-1                      */
+    int64_t step;       /* decode steps taken                                            */
+} ec_cache;
+
+/* Fills *c after validating: 2 <= budget <= cap, 0 <= len <= budget, 1 <= offset <= budget-1. */
+int ec_cache_init(ec_cache *c, void *Kc_dev, void *Vc_dev, int N, int H, int D, int cap,
+                  int len, int budget, int offset);
+
+size_t ec_decode_workspace(const ec_cache *c);
+
+/*
+ * One generation step (Sec. 3.3 "Output Generation"; Algorithm 1, last branch):
+ *   out = softmax(scale * q [Kc; k_new]^T) [Vc; v_new]      over len + 1 rows, per unit
+ * then the new row joins the cache. If the cache was already at its budget, the row that
+ * has exactly `offset` rows behind it (counting the new one) leaves: queue position
+ * len - offset, which is the paper's fixed truncation location. Physically the new row
+ * overwrites that row's slot; below budget it is appended at slot `len`.
+ *
+ *   q_dev, k_new_dev, v_new_dev  bf16 [N, H, D]                 (in)
+ *   out_dev                      bf16 [N, H, D]                 (out)
+ *   evicted_slot_host            physical slot that was overwritten, or -1 when the cache
+ *                                was below budget (host int, written before return)
+ *   slot_written_host            physical slot now holding the new row (may be NULL)
+ * Updates c->len, c->ring_head, c->step on success.
+ */
+int ec_decode_step(const void *q_dev, const void *k_new_dev, const void *v_new_dev,
+                   ec_cache *c, float scale, void *out_dev,
+                   int *evicted_slot_host, int *slot_written_host,
+                   void *ws_dev, size_t ws_bytes, void *stream);
+
+/*
+ * `steps` consecutive ec_decode_step calls issued from native code. Step s reads
+ * q/k_new/v_new at element offset s*N*H*D of the three [steps, N, H, D] arrays and writes
+ * out at the same offset. evicted_slots_host (may be NULL) receives `steps` ints.
+ */
+int ec_decode_steps(const void *q_dev, const void *k_new_dev, const void *v_new_dev, int steps,
+                    ec_cache *c, float scale, void *out_dev, int *evicted_slots_host,
+                    void *ws_dev, size_t ws_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EC_H_ */

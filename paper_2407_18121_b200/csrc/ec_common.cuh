@@ -1,0 +1,74 @@
+// Shared device helpers and internal launch declarations of the Elastic Cache library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "ec.h"
+
+namespace ec {
+
+constexpr int kStatusBytes = 256;   // status block at the head of an importance workspace
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Eight bf16 values held in one 16-byte vector -> eight floats.
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8])
+{
+    f[0] = bf16lo(v.x); f[1] = bf16hi(v.x);
+    f[2] = bf16lo(v.y); f[3] = bf16hi(v.y);
+    f[4] = bf16lo(v.z); f[5] = bf16hi(v.z);
+    f[6] = bf16lo(v.w); f[7] = bf16hi(v.w);
+}
+
+__device__ __forceinline__ uint32_t pack2(float a, float b)
+{
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);   // .x = a (low half), .y = b
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+__device__ __forceinline__ uint4 pack8(const float (&f)[8])
+{
+    uint4 v;
+    v.x = pack2(f[0], f[1]);
+    v.y = pack2(f[2], f[3]);
+    v.z = pack2(f[4], f[5]);
+    v.w = pack2(f[6], f[7]);
+    return v;
+}
+
+// Read-only streaming load (data never written by the running kernel).
+__device__ __forceinline__ uint4 ldg_stream(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ---- launchers implemented in the .cu files (all asynchronous on `stream`) ----
+cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out,
+                              int N, int H, int T, int D, float scale, void *ws, cudaStream_t stream);
+size_t importance_workspace_bytes(int N, int H, int T, int D);
+
+cudaError_t launch_select(const float *scores, int N, int H, int T, int n_keep, int population,
+                          int protect_ends, int32_t *anchor_pos, int32_t *bucket_len, float *mean_ws,
+                          cudaStream_t stream);
+cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
+                         int n_keep, void *Kc, void *Vc, int cap, cudaStream_t stream);
+
+int decode_splits(int units, int rows);
+cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
+                          int units, int D, int cap, int len, int write_slot, float scale, void *out,
+                          float *partials, int splits, cudaStream_t stream);
+
+}  // namespace ec
