@@ -1,0 +1,165 @@
+// Anchor selection (Sec. 3.3: the N_I positions with the highest importance, ascending)
+// as an exact radix select on fp32 bit patterns followed by an order-preserving compaction.
+#include "ec_common.cuh"
+
+namespace ec {
+
+namespace {
+
+constexpr int kSelThreads = 256;
+
+// Order-preserving map from fp32 to uint32 (larger float -> larger key).
+__device__ __forceinline__ uint32_t sort_key(float x)
+{
+    uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Layer-wise population: mean over the heads of a problem. scores [N,H,T] -> mean [N,T].
+__global__ void head_mean_kernel(const float *__restrict__ scores, float *__restrict__ mean, int H, int T)
+{
+    int n = blockIdx.y;
+    int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const float *s = scores + (size_t)n * H * T + t;
+    float acc = 0.f;
+    for (int h = 0; h < H; ++h) acc += s[(size_t)h * T];
+    mean[(size_t)n * T + t] = acc / (float)H;
+}
+
+// One CTA per selection unit. Dynamic shared memory: T keys + n_keep anchors.
+// `replicate` > 1 writes the same anchors for that many consecutive heads (layer-shared mode).
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(const float *__restrict__ scores, int T, int C, int protect_ends, int replicate,
+              int32_t *__restrict__ anchor_pos, int32_t *__restrict__ bucket_len)
+{
+    extern __shared__ uint32_t smem[];
+    uint32_t *keys = smem;
+    int32_t *anch = reinterpret_cast<int32_t *>(smem + T);
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t s_prefix, s_need;
+    __shared__ uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32];
+
+    const int tid = threadIdx.x;
+    const size_t unit = blockIdx.x;
+    const float *s = scores + unit * T;
+
+    for (int t = tid; t < T; t += kSelThreads) {
+        uint32_t k = sort_key(s[t]);
+        if (protect_ends && (t == 0 || (t == T - 1 && C >= 2))) k = 0xFFFFFFFFu;
+        keys[t] = k;
+    }
+    if (tid == 0) { s_prefix = 0; s_need = (uint32_t)C; }
+    __syncthreads();
+
+    // Four 8-bit digits, most significant first: find the C-th largest key.
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        hist[tid] = 0;                       // kSelThreads == 256 bins
+        __syncthreads();
+        const uint32_t prefix = s_prefix, need = s_need;
+        const uint32_t himask = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
+        for (int t = tid; t < T; t += kSelThreads) {
+            uint32_t k = keys[t];
+            if ((k & himask) == prefix) atomicAdd(&hist[(k >> shift) & 0xFF], 1u);
+        }
+        __syncthreads();
+        if (tid < 32) {
+            // lane l owns bins 255-8l .. 248-8l (descending); suffix-scan across lanes
+            uint32_t local[8], sum = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { local[i] = hist[255 - (tid * 8 + i)]; sum += local[i]; }
+            uint32_t incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (tid >= o) incl += v;
+            }
+            uint32_t before = incl - sum;    // keys in strictly higher bins than this lane's
+            if (before < need && need <= incl) {
+                uint32_t run = before;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (run < need && need <= run + local[i]) {
+                        s_prefix = prefix | ((uint32_t)(255 - (tid * 8 + i)) << shift);
+                        s_need = need - run;  // how many are still needed inside this bin
+                    }
+                    run += local[i];
+                }
+            }
+        }
+        __syncthreads();
+    }
+    const uint32_t thr = s_prefix;       // key of the C-th largest element
+    const uint32_t need_eq = s_need;     // how many keys equal to thr are taken (lowest positions)
+
+    // Ordered compaction: thread i owns the contiguous positions [i*ipt, (i+1)*ipt).
+    const int ipt = (T + kSelThreads - 1) / kSelThreads;
+    const int t0 = min(tid * ipt, T), t1 = min(t0 + ipt, T);
+    uint32_t gt = 0, eq = 0;
+    for (int t = t0; t < t1; ++t) {
+        uint32_t k = keys[t];
+        gt += (k > thr);
+        eq += (k == thr);
+    }
+    uint32_t gt_incl = gt, eq_incl = eq;
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t a = __shfl_up_sync(0xFFFFFFFFu, gt_incl, o);
+        uint32_t b = __shfl_up_sync(0xFFFFFFFFu, eq_incl, o);
+        if (lane >= o) { gt_incl += a; eq_incl += b; }
+    }
+    if (lane == 31) { warp_gt[warp] = gt_incl; warp_eq[warp] = eq_incl; }
+    __syncthreads();
+    uint32_t gt_before = gt_incl - gt, eq_before = eq_incl - eq;
+    for (int w = 0; w < warp; ++w) { gt_before += warp_gt[w]; eq_before += warp_eq[w]; }
+    for (int t = t0; t < t1; ++t) {
+        uint32_t k = keys[t];
+        if (k > thr) {
+            anch[gt_before + min(eq_before, need_eq)] = t;
+            ++gt_before;
+        } else if (k == thr) {
+            if (eq_before < need_eq) anch[gt_before + eq_before] = t;
+            ++eq_before;
+        }
+    }
+    __syncthreads();
+
+    for (int r = 0; r < replicate; ++r) {
+        int32_t *ap = anchor_pos + (unit * replicate + r) * C;
+        for (int k = tid; k < C; k += kSelThreads) ap[k] = anch[k];
+        if (bucket_len) {
+            // Eq. 2: bucket k spans floor((t_{k-1}+t_k)/2)+1 .. floor((t_k+t_{k+1})/2)
+            int32_t *bl = bucket_len + (unit * replicate + r) * C;
+            for (int k = tid; k < C; k += kSelThreads) {
+                int lo = (k == 0) ? 0 : ((anch[k - 1] + anch[k]) >> 1) + 1;
+                int hi = (k == C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
+                bl[k] = hi - lo + 1;
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_select(const float *scores, int N, int H, int T, int n_keep, int population,
+                          int protect_ends, int32_t *anchor_pos, int32_t *bucket_len, float *mean_ws,
+                          cudaStream_t stream)
+{
+    size_t smem = (size_t)(T + n_keep) * sizeof(uint32_t);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    if (population == EC_LAYER_SHARED) {
+        dim3 g((T + 255) / 256, N);
+        head_mean_kernel<<<g, 256, 0, stream>>>(scores, mean_ws, H, T);
+        select_kernel<<<N, kSelThreads, smem, stream>>>(mean_ws, T, n_keep, protect_ends, H, anchor_pos, bucket_len);
+    } else {
+        select_kernel<<<N * H, kSelThreads, smem, stream>>>(scores, T, n_keep, protect_ends, 1, anchor_pos, bucket_len);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace ec
