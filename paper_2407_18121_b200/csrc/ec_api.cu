@@ -1,0 +1,195 @@
+// C ABI of the library: argument validation, workspace layout and kernel sequencing.
+// Every step of the path runs in the CUDA kernels; nothing here computes on the host
+// beyond integer bookkeeping of the cache (which slot the next row goes to).
+#include "ec_common.cuh"
+
+#include <math.h>
+
+namespace {
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+
+constexpr int kMaxT = 16384;
+
+int check_shape(int N, int H, int T, int D)
+{
+    if (N < 1 || H < 1 || T < 1 || T > kMaxT) return EC_ERR_SHAPE;
+    if (D != 64 && D != 128) return EC_ERR_SHAPE;
+    if ((long long)N * H * T >= (1LL << 31)) return EC_ERR_SHAPE;
+    if ((long long)N * H >= (1LL << 24)) return EC_ERR_SHAPE;
+    return EC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *ec_status_string(int status)
+{
+    switch (status) {
+    case EC_OK: return "ok";
+    case EC_ERR_NULL: return "required pointer is NULL";
+    case EC_ERR_SHAPE: return "unsupported shape";
+    case EC_ERR_ALIGN: return "pointer not sufficiently aligned";
+    case EC_ERR_ARG: return "argument out of range";
+    case EC_ERR_WORKSPACE: return "workspace missing or too small";
+    case EC_ERR_CUDA: return "CUDA runtime error";
+    case EC_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+    }
+}
+
+int ec_keep_count(int T, double keep_ratio)
+{
+    if (T < 1 || !(keep_ratio >= 0.0 && keep_ratio <= 1.0)) return 0;
+    // Algorithm 1: del_num = int(seq_len - n * retained_fraction) with n = seq_len = T
+    int del = (int)((double)T - (double)T * keep_ratio);
+    if (del < 0) del = 0;
+    int keep = T - del;
+    if (keep < 1) keep = 1;
+    if (keep > T) keep = T;
+    return keep;
+}
+
+size_t ec_importance_workspace(int N, int H, int T, int D)
+{
+    if (check_shape(N, H, T, D) != EC_OK) return 0;
+    return ec::importance_workspace_bytes(N, H, T, D);
+}
+
+int ec_importance(const void *Q, const void *K, float *scores, float *lse, int N, int H, int T, int D,
+                  float scale, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!Q || !K || !scores) return EC_ERR_NULL;
+    int st = check_shape(N, H, T, D);
+    if (st != EC_OK) return st;
+    if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || (lse && !aligned(lse, 16))) return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    cudaError_t e = ec::launch_importance(Q, K, scores, lse, N, H, T, D, scale, ws, (cudaStream_t)stream);
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+int ec_device_status(void *ws, void *stream)
+{
+    if (!ws) return EC_ERR_NULL;
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, ws, sizeof word, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return EC_ERR_CUDA;
+    return word == 0 ? EC_OK : EC_ERR_TIMEOUT;
+}
+
+size_t ec_select_merge_workspace(int N, int H, int T, int D, int n_keep, int population)
+{
+    if (check_shape(N, H, T, D) != EC_OK || n_keep < 1 || n_keep > T) return 0;
+    // layer-shared mode keeps the head-averaged scores [N, T]; a minimum keeps the pointer non-null
+    size_t mean = (population == EC_LAYER_SHARED) ? round256((size_t)N * T * sizeof(float)) : 0;
+    return 256 + mean;
+}
+
+int ec_select_merge(const void *K, const void *V, const float *scores, int N, int H, int T, int D, int n_keep,
+                    int population, int protect_ends, void *Kc, void *Vc, int cap, int32_t *anchor_pos,
+                    int32_t *bucket_len, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!K || !V || !scores || !Kc || !Vc || !anchor_pos) return EC_ERR_NULL;
+    int st = check_shape(N, H, T, D);
+    if (st != EC_OK) return st;
+    if (n_keep < 1 || n_keep > T || cap < n_keep) return EC_ERR_ARG;
+    if (population != EC_PER_HEAD && population != EC_LAYER_SHARED) return EC_ERR_ARG;
+    if ((long long)N * H * cap >= (1LL << 31)) return EC_ERR_SHAPE;
+    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(scores, 4) ||
+        !aligned(anchor_pos, 4) || (bucket_len && !aligned(bucket_len, 4)))
+        return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < ec_select_merge_workspace(N, H, T, D, n_keep, population)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    float *mean_ws = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = ec::launch_select(scores, N, H, T, n_keep, population, protect_ends ? 1 : 0, anchor_pos,
+                                      bucket_len, mean_ws, s);
+    if (e != cudaSuccess) return EC_ERR_CUDA;
+    e = ec::launch_merge(K, V, anchor_pos, N * H, T, D, n_keep, Kc, Vc, cap, s);
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+int ec_cache_init(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, int cap, int len, int budget, int offset)
+{
+    if (!c || !Kc || !Vc) return EC_ERR_NULL;
+    if (N < 1 || H < 1 || (D != 64 && D != 128) || cap < 1) return EC_ERR_SHAPE;
+    if ((long long)N * H * cap >= (1LL << 31) || (long long)N * H >= (1LL << 24)) return EC_ERR_SHAPE;
+    if (!aligned(Kc, 16) || !aligned(Vc, 16)) return EC_ERR_ALIGN;
+    if (budget < 2 || budget > cap || len < 0 || len > budget) return EC_ERR_ARG;
+    if (offset < 1 || offset > budget - 1) return EC_ERR_ARG;
+    c->Kc = Kc; c->Vc = Vc;
+    c->N = N; c->H = H; c->D = D; c->cap = cap;
+    c->len = len; c->budget = budget; c->offset = offset;
+    c->ring_head = 0;
+    c->step = 0;
+    return EC_OK;
+}
+
+size_t ec_decode_workspace(const ec_cache *c)
+{
+    if (!c) return 0;
+    const int units = c->N * c->H;
+    const int splits = ec::decode_splits(units, c->cap + 1);
+    return 256 + round256((size_t)units * splits * (c->D + 2) * sizeof(float));
+}
+
+int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
+                   int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!q || !k_new || !v_new || !c || !out || !evicted_slot) return EC_ERR_NULL;
+    if (!c->Kc || !c->Vc) return EC_ERR_NULL;
+    if (c->budget < 2 || c->budget > c->cap || c->len < 0 || c->len > c->budget || c->offset < 1 ||
+        c->offset > c->budget - 1 || c->ring_head < 0 || c->ring_head >= c->offset)
+        return EC_ERR_ARG;
+    if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
+    if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16)) return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < ec_decode_workspace(c)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+
+    // Fixed-point elimination: at budget, queue position len - offset leaves. Rows before the
+    // ring never move, so that queue position is always the ring's oldest slot.
+    int slot, evicted;
+    if (c->len < c->budget) {
+        slot = c->len;
+        evicted = -1;
+    } else {
+        slot = c->budget - c->offset + c->ring_head;
+        evicted = slot;
+    }
+    const int units = c->N * c->H;
+    const int splits = ec::decode_splits(units, c->len + 1);
+    float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
+    cudaError_t e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, scale,
+                                      out, partials, splits, (cudaStream_t)stream);
+    if (e != cudaSuccess) return EC_ERR_CUDA;
+    if (evicted >= 0) c->ring_head = (c->ring_head + 1) % c->offset;
+    else c->len += 1;
+    c->step += 1;
+    *evicted_slot = evicted;
+    if (slot_written) *slot_written = slot;
+    return EC_OK;
+}
+
+int ec_decode_steps(const void *q, const void *k_new, const void *v_new, int steps, ec_cache *c, float scale,
+                    void *out, int *evicted_slots, void *ws, size_t ws_bytes, void *stream)
+{
+    if (steps < 0) return EC_ERR_ARG;
+    if (!c) return EC_ERR_NULL;
+    const size_t stride = (size_t)c->N * c->H * c->D * 2;   // bytes of one [N, H, D] bf16 step
+    for (int s = 0; s < steps; ++s) {
+        int ev = -1;
+        int st = ec_decode_step(static_cast<const char *>(q) + s * stride, static_cast<const char *>(k_new) + s * stride,
+                                static_cast<const char *>(v_new) + s * stride, c, scale,
+                                static_cast<char *>(out) + s * stride, &ev, nullptr, ws, ws_bytes, stream);
+        if (st != EC_OK) return st;
+        if (evicted_slots) evicted_slots[s] = ev;
+    }
+    return EC_OK;
+}
+
+}  // extern "C"
