@@ -1,0 +1,177 @@
+"""ctypes binding of libec.so: one Python function per C entry point, same names.
+
+Only argument marshalling happens here (tensor -> device pointer, shape -> ints, the
+current torch stream -> cudaStream_t). All arithmetic runs in the CUDA kernels. Tensors
+must live on the current CUDA device and be contiguous. There is no CPU fallback: if the
+library cannot be loaded, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libec.so")
+
+EC_OK = 0
+EC_PER_HEAD = 0
+EC_LAYER_SHARED = 1
+
+EXPORTS = (
+    "ec_status_string", "ec_keep_count",
+    "ec_importance_workspace", "ec_importance", "ec_device_status",
+    "ec_select_merge_workspace", "ec_select_merge",
+    "ec_cache_init", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
+)
+
+
+class EcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (ec_status {status})")
+
+
+class ec_cache(C.Structure):
+    """Mirror of the C struct ec_cache (host-side plain data)."""
+    _fields_ = [("Kc", C.c_void_p), ("Vc", C.c_void_p),
+                ("N", C.c_int), ("H", C.c_int), ("D", C.c_int), ("cap", C.c_int),
+                ("len", C.c_int), ("budget", C.c_int), ("offset", C.c_int),
+                ("ring_head", C.c_int), ("step", C.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libec.so (once). Raises if it has not been built: there is no fallback path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2407_18121_b200.build` "
+                          "(the CUDA library is the only implementation)")
+    L = C.CDLL(LIB_PATH)
+    vp, i, f, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
+    L.ec_status_string.restype = C.c_char_p
+    L.ec_status_string.argtypes = [i]
+    L.ec_keep_count.restype = i
+    L.ec_keep_count.argtypes = [i, C.c_double]
+    L.ec_importance_workspace.restype = sz
+    L.ec_importance_workspace.argtypes = [i, i, i, i]
+    L.ec_importance.restype = i
+    L.ec_importance.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
+    L.ec_device_status.restype = i
+    L.ec_device_status.argtypes = [vp, vp]
+    L.ec_select_merge_workspace.restype = sz
+    L.ec_select_merge_workspace.argtypes = [i, i, i, i, i, i]
+    L.ec_select_merge.restype = i
+    L.ec_select_merge.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, vp, vp, i, vp, vp, vp, sz, vp]
+    L.ec_cache_init.restype = i
+    L.ec_cache_init.argtypes = [C.POINTER(ec_cache), vp, vp, i, i, i, i, i, i, i]
+    L.ec_decode_workspace.restype = sz
+    L.ec_decode_workspace.argtypes = [C.POINTER(ec_cache)]
+    L.ec_decode_step.restype = i
+    L.ec_decode_step.argtypes = [vp, vp, vp, C.POINTER(ec_cache), f, vp, C.POINTER(i), C.POINTER(i), vp, sz, vp]
+    L.ec_decode_steps.restype = i
+    L.ec_decode_steps.argtypes = [vp, vp, vp, i, C.POINTER(ec_cache), f, vp, C.POINTER(i), vp, sz, vp]
+    _lib = L
+    return L
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("device tensors are required (the library has no host path)")
+    if not t.is_contiguous():
+        raise ValueError("tensors must be contiguous")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != EC_OK:
+        raise EcError(status, where)
+
+
+def status_string(status: int) -> str:
+    return lib().ec_status_string(int(status)).decode()
+
+
+def ec_keep_count(T: int, keep_ratio: float) -> int:
+    return int(lib().ec_keep_count(int(T), float(keep_ratio)))
+
+
+def ec_importance_workspace(N: int, H: int, T: int, D: int) -> int:
+    return int(lib().ec_importance_workspace(N, H, T, D))
+
+
+def ec_importance(Q: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, lse: Optional[torch.Tensor],
+                  scale: float, ws: torch.Tensor) -> None:
+    """Q, K: bf16 [N,H,T,D]; scores (out), lse (out, optional): fp32 [N,H,T]; ws: uint8 scratch."""
+    N, H, T, D = Q.shape
+    st = lib().ec_importance(_ptr(Q), _ptr(K), _ptr(scores), _ptr(lse), N, H, T, D, float(scale),
+                             _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_importance")
+
+
+def ec_device_status(ws: torch.Tensor) -> int:
+    return int(lib().ec_device_status(_ptr(ws), _stream()))
+
+
+def ec_select_merge_workspace(N: int, H: int, T: int, D: int, n_keep: int, population: int) -> int:
+    return int(lib().ec_select_merge_workspace(N, H, T, D, n_keep, population))
+
+
+def ec_select_merge(K: torch.Tensor, V: torch.Tensor, scores: torch.Tensor, n_keep: int, population: int,
+                    protect_ends: bool, Kc: torch.Tensor, Vc: torch.Tensor, anchor_pos: torch.Tensor,
+                    bucket_len: Optional[torch.Tensor], ws: torch.Tensor) -> None:
+    """K, V: bf16 [N,H,T,D]; scores fp32 [N,H,T]; Kc, Vc (out): bf16 [N,H,cap,D];
+    anchor_pos (out), bucket_len (out, optional): int32 [N,H,n_keep]."""
+    N, H, T, D = K.shape
+    cap = Kc.shape[2]
+    st = lib().ec_select_merge(_ptr(K), _ptr(V), _ptr(scores), N, H, T, D, int(n_keep), int(population),
+                               int(bool(protect_ends)), _ptr(Kc), _ptr(Vc), cap, _ptr(anchor_pos),
+                               _ptr(bucket_len), _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_select_merge")
+
+
+def ec_cache_init(Kc: torch.Tensor, Vc: torch.Tensor, length: int, budget: int, offset: int) -> ec_cache:
+    """Describe a compacted cache held in Kc, Vc: bf16 [N,H,cap,D] with `length` valid rows."""
+    N, H, cap, D = Kc.shape
+    c = ec_cache()
+    st = lib().ec_cache_init(C.byref(c), _ptr(Kc), _ptr(Vc), N, H, D, cap, int(length), int(budget), int(offset))
+    _check(st, "ec_cache_init")
+    return c
+
+
+def ec_decode_workspace(cache: ec_cache) -> int:
+    return int(lib().ec_decode_workspace(C.byref(cache)))
+
+
+def ec_decode_step(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, cache: ec_cache, scale: float,
+                   out: torch.Tensor, ws: torch.Tensor):
+    """q, k_new, v_new: bf16 [N,H,D]; out (out): bf16 [N,H,D].
+    Returns (evicted physical slot or -1, slot that now holds the new row)."""
+    ev, sl = C.c_int(-1), C.c_int(-1)
+    st = lib().ec_decode_step(_ptr(q), _ptr(k_new), _ptr(v_new), C.byref(cache), float(scale), _ptr(out),
+                              C.byref(ev), C.byref(sl), _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_decode_step")
+    return ev.value, sl.value
+
+
+def ec_decode_steps(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, cache: ec_cache, scale: float,
+                    out: torch.Tensor, ws: torch.Tensor, want_slots: bool = False):
+    """q, k_new, v_new, out: bf16 [steps,N,H,D]. Issues all steps from native code."""
+    steps = q.shape[0]
+    slots = (C.c_int * steps)() if want_slots else None
+    st = lib().ec_decode_steps(_ptr(q), _ptr(k_new), _ptr(v_new), steps, C.byref(cache), float(scale), _ptr(out),
+                               slots, _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_decode_steps")
+    return list(slots) if want_slots else None

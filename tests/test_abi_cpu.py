@@ -1,0 +1,95 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every
+declared symbol, and rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from oracle import ec_oracle as orc
+from paper_2407_18121_b200 import binding as ec
+from paper_2407_18121_b200 import build as ecbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    ecbuild.build()
+    return ec.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "ec.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ec_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = _declared()
+    assert len(names) >= 11
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in ec.h but not exported"
+    assert sorted(ec.EXPORTS) == names
+
+
+def test_keep_count_matches_oracle_rule(L):
+    for T in (1, 2, 7, 100, 256, 640, 1024, 2048, 8192, 16384):
+        for r in (0.0, 0.05, 0.1, 0.2, 0.25, 0.3, 0.5, 0.7, 0.75, 0.9, 1.0):
+            assert ec.ec_keep_count(T, r) == orc.keep_count(T, r), (T, r)
+    assert ec.ec_keep_count(0, 0.5) == 0 and ec.ec_keep_count(10, 1.5) == 0
+
+
+def test_status_strings(L):
+    seen = {ec.status_string(s) for s in range(8)}
+    assert len(seen) == 8 and ec.status_string(99) == "unknown status"
+
+
+def test_importance_rejects_bad_arguments_on_the_host(L):
+    p = 0x10000  # fake, aligned, never dereferenced: every case below fails validation first
+    f = L.ec_importance
+    assert f(None, p, p, None, 1, 1, 16, 64, 1.0, p, 1 << 20, None) == 1          # NULL
+    assert f(p, p, p, None, 1, 1, 16, 96, 1.0, p, 1 << 20, None) == 2             # D
+    assert f(p, p, p, None, 1, 1, 0, 64, 1.0, p, 1 << 20, None) == 2              # T
+    assert f(p + 2, p, p, None, 1, 1, 16, 64, 1.0, p, 1 << 20, None) == 3         # alignment
+    assert f(p, p, p, None, 1, 1, 16, 64, -1.0, p, 1 << 20, None) == 4            # scale
+    assert f(p, p, p, None, 1, 1, 16, 64, 1.0, None, 0, None) == 5                # workspace
+    assert f(p, p, p, None, 1, 1, 16, 64, 1.0, p, 16, None) == 5
+    assert L.ec_importance_workspace(1, 1, 16, 64) >= 256 + 64
+    assert L.ec_importance_workspace(1, 1, 16, 100) == 0
+
+
+def test_select_merge_rejects_bad_arguments_on_the_host(L):
+    p = 0x10000
+    f = L.ec_select_merge
+    ok_ws = 1 << 20
+    assert f(p, p, None, 1, 1, 16, 64, 8, 0, 0, p, p, 8, p, None, p, ok_ws, None) == 1
+    assert f(p, p, p, 1, 1, 16, 64, 0, 0, 0, p, p, 8, p, None, p, ok_ws, None) == 4    # n_keep
+    assert f(p, p, p, 1, 1, 16, 64, 17, 0, 0, p, p, 32, p, None, p, ok_ws, None) == 4
+    assert f(p, p, p, 1, 1, 16, 64, 8, 0, 0, p, p, 7, p, None, p, ok_ws, None) == 4    # cap < n_keep
+    assert f(p, p, p, 1, 1, 16, 64, 8, 2, 0, p, p, 8, p, None, p, ok_ws, None) == 4    # population
+    assert f(p, p, p, 1, 1, 16, 64, 8, 0, 0, p + 8, p, 8, p, None, p, ok_ws, None) == 3
+    assert f(p, p, p, 1, 1, 16, 64, 8, 0, 0, p, p, 8, p, None, None, 0, None) == 5
+
+
+def test_cache_init_and_decode_validation(L):
+    p = 0x10000
+    c = ec.ec_cache()
+    init = L.ec_cache_init
+    assert init(C.byref(c), p, p, 2, 3, 64, 16, 8, 8, 4) == 0
+    assert (c.N, c.H, c.D, c.cap, c.len, c.budget, c.offset, c.ring_head, c.step) == (2, 3, 64, 16, 8, 8, 4, 0, 0)
+    assert init(C.byref(c), None, p, 2, 3, 64, 16, 8, 8, 4) == 1
+    assert init(C.byref(c), p, p, 2, 3, 48, 16, 8, 8, 4) == 2
+    assert init(C.byref(c), p, p, 2, 3, 64, 16, 9, 8, 4) == 4      # len > budget
+    assert init(C.byref(c), p, p, 2, 3, 64, 16, 8, 17, 4) == 4     # budget > cap
+    assert init(C.byref(c), p, p, 2, 3, 64, 16, 8, 8, 0) == 4      # offset < 1
+    assert init(C.byref(c), p, p, 2, 3, 64, 16, 8, 8, 8) == 4      # offset > budget - 1
+    assert init(C.byref(c), p, p, 2, 3, 64, 16, 8, 8, 4) == 0
+    ev = C.c_int(0)
+    step = L.ec_decode_step
+    assert step(None, p, p, C.byref(c), 1.0, p, C.byref(ev), None, p, 1 << 20, None) == 1
+    assert step(p, p, p, C.byref(c), 0.0, p, C.byref(ev), None, p, 1 << 20, None) == 4
+    assert step(p, p + 4, p, C.byref(c), 1.0, p, C.byref(ev), None, p, 1 << 20, None) == 3
+    assert step(p, p, p, C.byref(c), 1.0, p, C.byref(ev), None, None, 0, None) == 5
+    assert (c.len, c.ring_head, c.step) == (8, 0, 0)               # failed calls leave the state alone
+    assert L.ec_decode_workspace(C.byref(c)) >= 256
