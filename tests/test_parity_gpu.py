@@ -1,0 +1,350 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded bf16 inputs. Oracle inputs never come from the GPU: stage tests feed the
+GPU with the oracle's own intermediate results."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ec_oracle as orc
+from paper_2407_18121_b200 import binding as ec
+from paper_2407_18121_b200 import workloads as wl
+from helpers import (SCORE_RTOL, Guarded, assert_bf16_close, assert_rel_close, dev_bf16, host_bits, host_f64,
+                     scratch)
+
+pytestmark = pytest.mark.gpu
+
+
+def rand_bits(rng, shape, sigma=1.0):
+    return wl.to_bf16_bits(rng.standard_normal(shape).astype(np.float32) * np.float32(sigma))
+
+
+# ---------------------------------------------------------------- stage runners
+
+def gpu_importance(Qb, Kb, scale, want_lse=True):
+    N, H, T, D = Qb.shape
+    Q, K = dev_bf16(Qb), dev_bf16(Kb)
+    scores = Guarded((N, H, T), torch.float32, fill=float("nan"))
+    lse = Guarded((N, H, T), torch.float32, fill=float("nan")) if want_lse else None
+    ws = scratch(ec.ec_importance_workspace(N, H, T, D))
+    ec.ec_importance(Q, K, scores.t, lse.t if lse else None, scale, ws)
+    assert ec.ec_device_status(ws) == ec.EC_OK
+    scores.check("scores")
+    if lse:
+        lse.check("lse")
+    return scores.t, (lse.t if lse else None)
+
+
+def gpu_select_merge(Kb, Vb, scores_f32, n_keep, population, protect, cap=None):
+    N, H, T, D = Kb.shape
+    cap = n_keep if cap is None else cap
+    K, V = dev_bf16(Kb), dev_bf16(Vb)
+    s = torch.from_numpy(np.ascontiguousarray(scores_f32, np.float32)).cuda()
+    Kc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
+    Vc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
+    anchors = Guarded((N, H, n_keep), torch.int32, fill=-7)
+    blen = Guarded((N, H, n_keep), torch.int32, fill=-7)
+    ws = scratch(ec.ec_select_merge_workspace(N, H, T, D, n_keep, population))
+    ec.ec_select_merge(K, V, s, n_keep, population, protect, Kc.t, Vc.t, anchors.t, blen.t, ws)
+    for g, name in ((Kc, "Kc"), (Vc, "Vc"), (anchors, "anchor_pos"), (blen, "bucket_len")):
+        g.check(name)
+    return Kc.t, Vc.t, anchors.t, blen.t
+
+
+def check_anchor_sets(gpu_anchors, oracle_anchors, scores64, n_keep, protect, band=1e-4):
+    """Index sets must be equal, except for positions whose score lies within `band` (relative)
+    of the n_keep-th largest score: there either choice is a correct answer."""
+    ga = gpu_anchors.cpu().numpy()
+    T = scores64.shape[-1]
+    ga2 = ga.reshape(-1, n_keep)
+    oa2 = oracle_anchors.reshape(-1, n_keep)
+    sc2 = scores64.reshape(-1, T)
+    exact = 0
+    for u in range(ga2.shape[0]):
+        assert (np.diff(ga2[u]) > 0).all(), "anchors must be strictly ascending"
+        assert ga2[u].min() >= 0 and ga2[u].max() < T
+        if (ga2[u] == oa2[u]).all():
+            exact += 1
+            continue
+        s = sc2[u].copy()
+        if protect:
+            s[0] = np.inf
+            if n_keep >= 2:
+                s[-1] = np.inf
+        kth = np.sort(s)[::-1][n_keep - 1]
+        diff = np.setxor1d(ga2[u], oa2[u])
+        assert (np.abs(s[diff] - kth) <= band * abs(kth)).all(), \
+            f"unit {u}: anchor sets differ outside the tie band at positions {diff}"
+    return exact, ga2.shape[0]
+
+
+# ---------------------------------------------------------------- importance
+
+@pytest.mark.parametrize("N,H,T,D", [(1, 1, 1, 64), (1, 2, 2, 128), (2, 2, 127, 64), (1, 3, 129, 128),
+                                     (1, 2, 255, 128), (2, 1, 256, 64), (1, 2, 640, 128), (1, 1, 300, 64)])
+def test_importance_random(N, H, T, D):
+    rng = np.random.default_rng(T * 7 + D)
+    Qb, Kb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    scale = 1.0 / math.sqrt(D)
+    want, want_lse = orc.importance(Qb, Kb, scale)
+    got, got_lse = gpu_importance(Qb, Kb, scale)
+    assert_rel_close(got, want, SCORE_RTOL, what="scores")
+    assert_rel_close(got_lse, want_lse, 1e-3, atol=1e-3, what="lse")
+    np.testing.assert_allclose(host_f64(got).sum(-1), T, rtol=1e-3)      # rows of A sum to one
+
+
+def test_importance_peaked_logits_and_no_lse_output():
+    # large logits: the row maximum must be subtracted or exp overflows
+    rng = np.random.default_rng(3)
+    Qb, Kb = rand_bits(rng, (1, 2, 200, 128), 3.0), rand_bits(rng, (1, 2, 200, 128), 3.0)
+    want, _ = orc.importance(Qb, Kb, 1.0)
+    got, none = gpu_importance(Qb, Kb, 1.0, want_lse=False)
+    assert none is None
+    assert_rel_close(got, want, SCORE_RTOL, atol=1e-30, what="scores (peaked)")
+
+
+@pytest.mark.parametrize("name", ["tiny", "llava7b_b1", "long8k"])
+def test_importance_on_workload_recipes(name):
+    w = wl.WORKLOADS[name]
+    if name == "llava7b_b1":
+        Qb, Kb, _ = wl.prompt(w, [0, 31])
+        Qb, Kb = Qb[:, :4], Kb[:, :4]
+    elif name == "long8k":
+        Qb, Kb, _ = wl.prompt(w, [5])
+        Qb, Kb = Qb[:, :2, :1536], Kb[:, :2, :1536]      # several tiles of the recipe, oracle-sized
+    else:
+        Qb, Kb, _ = wl.prompt(w)
+    Qb, Kb = np.ascontiguousarray(Qb), np.ascontiguousarray(Kb)
+    want, want_lse = orc.importance(Qb, Kb, w.scale)
+    got, got_lse = gpu_importance(Qb, Kb, w.scale)
+    assert_rel_close(got, want, SCORE_RTOL, what=f"scores[{name}]")
+    assert_rel_close(got_lse, want_lse, 1e-3, atol=1e-3, what=f"lse[{name}]")
+
+
+def test_importance_is_deterministic():
+    rng = np.random.default_rng(8)
+    Qb, Kb = rand_bits(rng, (2, 3, 333, 128)), rand_bits(rng, (2, 3, 333, 128))
+    a, _ = gpu_importance(Qb, Kb, 0.1)
+    b, _ = gpu_importance(Qb, Kb, 0.1)
+    assert torch.equal(a, b)
+
+
+# ---------------------------------------------------------------- selection + merge
+
+@pytest.mark.parametrize("population", [ec.EC_PER_HEAD, ec.EC_LAYER_SHARED])
+@pytest.mark.parametrize("protect", [False, True])
+@pytest.mark.parametrize("N,H,T,D,n_keep", [(1, 1, 1, 64, 1), (1, 2, 2, 64, 1), (2, 3, 130, 128, 65),
+                                            (1, 4, 257, 64, 26), (2, 2, 640, 128, 320), (1, 2, 1000, 128, 1),
+                                            (1, 2, 300, 128, 299), (1, 1, 2048, 128, 205)])
+def test_select_merge_from_oracle_scores(N, H, T, D, n_keep, population, protect):
+    rng = np.random.default_rng(T + n_keep)
+    Kb, Vb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    # heavy-tailed positive scores, as column sums of attention are; fp32-exact so both sides rank
+    # the very same numbers
+    s32 = (rng.random((N, H, T)) ** 4 * 5 + 1e-3).astype(np.float32)
+    s64 = s32.astype(np.float64)
+    if population == ec.EC_LAYER_SHARED:
+        rank64 = np.repeat(orc.layer_mean(s64)[:, None, :], H, axis=1)
+    else:
+        rank64 = s64
+    want_anchors = orc.select(rank64, n_keep, protect)
+    Kc, Vc, anchors, blen = gpu_select_merge(Kb, Vb, s32, n_keep, population, protect)
+    exact, total = check_anchor_sets(anchors, want_anchors, rank64, n_keep, protect)
+    if population == ec.EC_PER_HEAD:
+        assert exact == total                       # same fp32 numbers on both sides: bit-exact sets
+    ga = anchors.cpu().numpy()
+    if population == ec.EC_LAYER_SHARED:
+        assert (ga == ga[:, :1]).all()              # every head of a problem shares the anchors
+    lo, hi = orc.buckets(ga, T)                     # merge is checked on the anchor set the GPU chose
+    np.testing.assert_array_equal(blen.cpu().numpy(), hi - lo + 1)
+    assert_bf16_close(Kc, orc.merge(Kb, lo, hi), "merged K")
+    assert_bf16_close(Vc, orc.merge(Vb, lo, hi), "merged V")
+
+
+def test_keep_everything_is_the_identity():
+    rng = np.random.default_rng(21)
+    N, H, T, D = 2, 3, 193, 128
+    Kb, Vb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    s32 = rng.random((N, H, T)).astype(np.float32)
+    Kc, Vc, anchors, blen = gpu_select_merge(Kb, Vb, s32, T, ec.EC_PER_HEAD, True)
+    np.testing.assert_array_equal(host_bits(Kc), Kb)          # bit-identical cache
+    np.testing.assert_array_equal(host_bits(Vc), Vb)
+    assert (anchors.cpu().numpy() == np.arange(T)).all() and (blen.cpu().numpy() == 1).all()
+
+
+def test_exact_ties_go_to_the_lower_position():
+    N, H, T, D = 1, 2, 96, 64
+    rng = np.random.default_rng(5)
+    Kb, Vb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    s32 = rng.integers(1, 4, size=(N, H, T)).astype(np.float32)       # only three distinct values
+    for n_keep in (1, 10, 48, 95):
+        want = orc.select(s32.astype(np.float64), n_keep, False)
+        _, _, anchors, _ = gpu_select_merge(Kb, Vb, s32, n_keep, ec.EC_PER_HEAD, False)
+        np.testing.assert_array_equal(anchors.cpu().numpy(), want)
+
+
+def test_cap_larger_than_keep_leaves_tail_rows_untouched():
+    rng = np.random.default_rng(6)
+    N, H, T, D, n_keep, cap = 1, 2, 100, 128, 30, 47
+    Kb, Vb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    s32 = rng.random((N, H, T)).astype(np.float32)
+    Kc, Vc, anchors, _ = gpu_select_merge(Kb, Vb, s32, n_keep, ec.EC_PER_HEAD, False, cap=cap)
+    assert torch.isnan(Kc[:, :, n_keep:].float()).all() and torch.isnan(Vc[:, :, n_keep:].float()).all()
+    lo, hi = orc.buckets(anchors.cpu().numpy(), T)
+    assert_bf16_close(Kc[:, :, :n_keep].contiguous(), orc.merge(Kb, lo, hi), "merged K")
+
+
+# ---------------------------------------------------------------- decode + fixed-point eviction
+
+def run_decode_case(N, H, D, C, cap, len0, offset, steps, scale, seed, sigma_k=1.0):
+    """Cache contents come from the oracle side (random bf16 rows); both sides run `steps` steps."""
+    rng = np.random.default_rng(seed)
+    K0b, V0b = rand_bits(rng, (N, H, len0, D), sigma_k), rand_bits(rng, (N, H, len0, D))
+    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=max(C, len0) + 1)
+    Kc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
+    Vc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
+    Kc.t[:, :, :len0] = dev_bf16(K0b)
+    Vc.t[:, :, :len0] = dev_bf16(V0b)
+    cache = ec.ec_cache_init(Kc.t, Vc.t, len0, C, offset)
+    ws = scratch(ec.ec_decode_workspace(cache))
+    slot_ids = list(range(len0)) + [-1] * (cap - len0)        # identity held by each physical slot
+    evictions = 0
+    for s in range(steps):
+        qb, kb, vb = rand_bits(rng, (N, H, D)), rand_bits(rng, (N, H, D), sigma_k), rand_bits(rng, (N, H, D))
+        len_before = cache.len
+        want, pos, ident = queue.step(qb, kb, vb, scale, policy=orc.POLICY_FIXED, budget=C, offset=offset)
+        out = Guarded((N, H, D), torch.bfloat16, fill=float("nan"))
+        ev, slot = ec.ec_decode_step(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), cache, scale, out.t, ws)
+        out.check("out")
+        assert_bf16_close(out.t, want, f"decode out, step {s}")
+        if len_before < C:
+            assert ev == -1 and pos == -1 and slot == len_before
+        else:
+            assert pos == C - offset                                 # the fixed truncation location
+            assert ev == slot == (C - offset) + (evictions % offset)  # ring of `offset` slots
+            assert slot_ids[ev] == ident                              # the same row leaves on both sides
+            evictions += 1
+        slot_ids[slot] = queue.next_id - 1
+        assert cache.len == queue.len and cache.step == s + 1
+        assert sorted(slot_ids[:cache.len]) == sorted(queue.identities().tolist())
+    Kc.check("Kc")
+    Vc.check("Vc")
+    # the device cache holds exactly the oracle queue's rows (as a set; order is physical)
+    Kdev = host_f64(Kc.t[:, :, :cache.len])
+    ids = queue.identities().tolist()
+    for j, ident in enumerate(ids):
+        phys = slot_ids.index(ident)
+        np.testing.assert_array_equal(Kdev[:, :, phys], queue.K[:, j].reshape(N, H, D))
+    return cache
+
+
+@pytest.mark.parametrize("N,H,D,C,offset,steps", [
+    (1, 8, 64, 128, 16, 40),        # few units: the rows of a unit are split over several CTAs
+    (1, 2, 128, 70, 25, 60),        # the paper's recent distance of 25
+    (20, 32, 128, 96, 16, 20),      # many units: one CTA per unit
+    (3, 5, 64, 33, 1, 5),           # offset 1: only the newest row is protected
+    (2, 2, 128, 9, 8, 20),          # offset = budget - 1: only the first row is protected
+])
+def test_decode_at_budget(N, H, D, C, offset, steps):
+    run_decode_case(N, H, D, C, C, C, offset, steps, 1.0 / math.sqrt(D), seed=C + offset)
+
+
+def test_decode_below_budget_grows_then_evicts():
+    cache = run_decode_case(2, 4, 128, 40, 48, 30, 6, 25, 0.1, seed=77)
+    assert cache.len == 40
+
+
+def test_decode_from_empty_cache():
+    # len 0: the first step attends to the new row only, so out == v_new exactly
+    N, H, D = 1, 3, 64
+    rng = np.random.default_rng(1)
+    Kc = torch.zeros((N, H, 8, D), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    cache = ec.ec_cache_init(Kc, Vc, 0, 4, 2)
+    ws = scratch(ec.ec_decode_workspace(cache))
+    qb, kb, vb = rand_bits(rng, (N, H, D)), rand_bits(rng, (N, H, D)), rand_bits(rng, (N, H, D))
+    out = torch.empty((N, H, D), dtype=torch.bfloat16, device="cuda")
+    ev, slot = ec.ec_decode_step(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), cache, 1.0, out, ws)
+    assert (ev, slot, cache.len) == (-1, 0, 1)
+    np.testing.assert_array_equal(host_bits(out), vb)
+    np.testing.assert_array_equal(host_bits(Kc[:, :, 0]), kb)
+
+
+def test_decode_peaked_logits():
+    run_decode_case(1, 4, 128, 64, 64, 64, 16, 6, 1.0, seed=9, sigma_k=3.0)
+
+
+def test_decode_steps_native_loop_matches_single_steps():
+    rng = np.random.default_rng(4)
+    N, H, D, C, d, S = 2, 3, 128, 50, 16, 37
+    K0, V0 = dev_bf16(rand_bits(rng, (N, H, C, D))), dev_bf16(rand_bits(rng, (N, H, C, D)))
+    q, k, v = (dev_bf16(rand_bits(rng, (S, N, H, D))) for _ in range(3))
+    Ka, Va, Kb_, Vb_ = K0.clone(), V0.clone(), K0.clone(), V0.clone()
+    ca, cb = ec.ec_cache_init(Ka, Va, C, C, d), ec.ec_cache_init(Kb_, Vb_, C, C, d)
+    ws = scratch(ec.ec_decode_workspace(ca))
+    out_a = torch.empty((S, N, H, D), dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty_like(out_a)
+    slots_a = [ec.ec_decode_step(q[s], k[s], v[s], ca, 0.2, out_a[s], ws)[0] for s in range(S)]
+    slots_b = ec.ec_decode_steps(q, k, v, cb, 0.2, out_b, ws, want_slots=True)
+    assert slots_a == slots_b == [(C - d) + (s % d) for s in range(S)]
+    assert torch.equal(out_a, out_b) and torch.equal(Ka, Kb_) and torch.equal(Va, Vb_)
+    assert (cb.len, cb.ring_head, cb.step) == (C, S % d, S)
+
+
+# ---------------------------------------------------------------- the whole path
+
+@pytest.mark.parametrize("name,population", [("tiny", ec.EC_PER_HEAD), ("tiny", ec.EC_LAYER_SHARED),
+                                             ("llava7b_b1", ec.EC_PER_HEAD)])
+def test_whole_path_on_workload(name, population):
+    """importance -> select/merge -> decode loop entirely on the GPU, against the oracle chain."""
+    w = wl.WORKLOADS[name]
+    if name == "llava7b_b1":
+        problems, heads, steps = [7], 3, 24
+    else:
+        problems, heads, steps = [0], w.heads, w.decode_steps
+    Qb, Kb, Vb = (np.ascontiguousarray(x[:, :heads]) for x in wl.prompt(w, problems))
+    N, H, T, D = Qb.shape
+    C = ec.ec_keep_count(T, w.keep_ratio)
+    assert C == orc.keep_count(T, w.keep_ratio)
+
+    o_scores, _ = orc.importance(Qb, Kb, w.scale)
+    rank = o_scores if population == ec.EC_PER_HEAD else np.repeat(orc.layer_mean(o_scores)[:, None], H, 1)
+    o_anchors = orc.select(rank, C, True)
+
+    Q, K, V = dev_bf16(Qb), dev_bf16(Kb), dev_bf16(Vb)
+    scores = torch.empty((N, H, T), dtype=torch.float32, device="cuda")
+    ws_i = scratch(ec.ec_importance_workspace(N, H, T, D))
+    ec.ec_importance(Q, K, scores, None, w.scale, ws_i)
+    Kc = torch.empty((N, H, C, D), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.empty_like(Kc)
+    anchors = torch.empty((N, H, C), dtype=torch.int32, device="cuda")
+    ws_m = scratch(ec.ec_select_merge_workspace(N, H, T, D, C, population))
+    ec.ec_select_merge(K, V, scores, C, population, True, Kc, Vc, anchors, None, ws_m)
+    assert_rel_close(scores, o_scores, SCORE_RTOL, what="scores")
+    check_anchor_sets(anchors, o_anchors, rank, C, True)
+    if name == "tiny" and population == ec.EC_PER_HEAD:
+        # the four boosted keys of every head draw most of the attention: all must be anchors
+        knorm = np.linalg.norm(wl.bf16_bits_to_f64(Kb), axis=-1)
+        for h in range(H):
+            heavy = np.argsort(knorm[0, h])[-4:]
+            assert np.isin(heavy, anchors[0, h].cpu().numpy()).all()
+
+    ga = anchors.cpu().numpy()
+    lo, hi = orc.buckets(ga, T)
+    o_Kc, o_Vc = orc.merge(Kb, lo, hi), orc.merge(Vb, lo, hi)
+    assert_bf16_close(Kc, o_Kc, "merged K")
+    assert_bf16_close(Vc, o_Vc, "merged V")
+
+    # the oracle decodes from its own merged rows, rounded to bf16 as the cache stores them
+    queue = orc.DecodeQueue(orc.widen_bf16(orc.round_bf16(o_Kc)), orc.widen_bf16(orc.round_bf16(o_Vc)), cap=C + 1)
+    cache = ec.ec_cache_init(Kc, Vc, C, C, w.offset)
+    ws_d = scratch(ec.ec_decode_workspace(cache))
+    out = torch.empty((N, H, D), dtype=torch.bfloat16, device="cuda")
+    for s in range(steps):
+        qb, kb, vb = (np.ascontiguousarray(x[:, :heads]) for x in wl.decode_step_inputs(w, s, problems))
+        want, pos, _ = queue.step(qb, kb, vb, w.scale, policy=orc.POLICY_FIXED, budget=C, offset=w.offset)
+        ev, _ = ec.ec_decode_step(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), cache, w.scale, out, ws_d)
+        assert ev == (C - w.offset) + (s % w.offset) and pos == C - w.offset
+        assert_bf16_close(out, want, f"decode out, step {s}")
+    assert cache.len == C
