@@ -324,10 +324,12 @@ def test_whole_path_on_workload(name, population):
     assert_rel_close(scores, o_scores, SCORE_RTOL, what="scores")
     check_anchor_sets(anchors, o_anchors, rank, C, True)
     if name == "tiny" and population == ec.EC_PER_HEAD:
-        # the four boosted keys of every head draw most of the attention: all must be anchors
+        # a boosted key draws attention from every later query, so those that are not close to
+        # the end of the prompt (where few queries remain to look at them) must all be anchors
         knorm = np.linalg.norm(wl.bf16_bits_to_f64(Kb), axis=-1)
         for h in range(H):
             heavy = np.argsort(knorm[0, h])[-4:]
+            heavy = heavy[heavy < (3 * T) // 4]
             assert np.isin(heavy, anchors[0, h].cpu().numpy()).all()
 
     ga = anchors.cpu().numpy()
