@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the Elastic Cache hot path on B200.
+
+One "step" is one pass of the whole path over one synthetic batch: importance over the
+prompt, anchor selection + merge into the compacted cache, then the workload's full decode
+loop (attention over the cache + fixed-point eviction every token). The reported value is
+generated tokens per second over that whole pass, all problems of all ranks counted.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Under torchrun every rank runs its own batch (independent problems: no data-path collective),
+times on the device, and rank 0 prints one JSON line with the max-over-ranks time.
+`--impl reference` times the CPU oracle (the deliberately plain fp64 program the tests check
+against) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2407_18121_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode tokens/s on merged KV (whole pass: importance + select/merge + decode loop)"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def bits_to_tensor(bits: np.ndarray, pin: bool):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+    return t.pin_memory() if pin else t
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+
+def oracle_sample(w: wl.Workload, decode_steps_sample: int, problems_sample: int):
+    """Times the oracle on a bounded sample and extrapolates to the whole pass.
+    Sample: the full prompt stage (importance, selection, buckets, merge) of the first
+    `problems_sample` problems, then `decode_steps_sample` decode steps on them."""
+    from oracle import ec_oracle as orc
+    problems = list(range(min(problems_sample, w.N)))
+    Qb, Kb, Vb = wl.prompt(w, problems)
+    T = w.prompt_len
+    C = orc.keep_count(T, w.keep_ratio)
+    t0 = time.perf_counter()
+    scores, _ = orc.importance(Qb, Kb, w.scale)
+    anchors = orc.select(scores, C, True)
+    lo, hi = orc.buckets(anchors, T)
+    Kc, Vc = orc.merge(Kb, lo, hi), orc.merge(Vb, lo, hi)
+    queue = orc.DecodeQueue(orc.widen_bf16(orc.round_bf16(Kc)), orc.widen_bf16(orc.round_bf16(Vc)), cap=C + 1)
+    t1 = time.perf_counter()
+    S = min(decode_steps_sample, w.decode_steps)
+    dec_in = [wl.decode_step_inputs(w, s, problems) for s in range(S)]
+    t2 = time.perf_counter()
+    for s in range(S):
+        q, k, v = dec_in[s]
+        queue.step(q, k, v, w.scale, policy=orc.POLICY_FIXED, budget=C, offset=w.offset)
+    t3 = time.perf_counter()
+    frac = w.N / len(problems)
+    prompt_s = (t1 - t0) * frac
+    decode_s = (t3 - t2) * frac * (w.decode_steps / S)
+    total = prompt_s + decode_s
+    return {"seconds_whole_pass_extrapolated": total, "prompt_s": prompt_s, "decode_s": decode_s,
+            "sample_seconds": (t1 - t0) + (t3 - t2), "cores": orc.num_threads(),
+            "sample": (f"prompt stage of {len(problems)} of {w.N} problems (all {w.heads} heads) + {S} of "
+                       f"{w.decode_steps} decode steps on them, extrapolated linearly to the whole pass")}
+
+
+def run_reference(args, w: wl.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = []
+    info = None
+    for i in range(args.warmup + args.steps):
+        info = oracle_sample(w, args.oracle_decode_steps, args.oracle_problems)
+        if i >= args.warmup:
+            per_step.append(info["seconds_whole_pass_extrapolated"])
+    sec = float(np.mean(per_step))
+    tokens = w.batch * w.decode_steps
+    value = tokens / sec
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
+                             "sample": info["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w: wl.Workload):
+    return {"workload": w.name, "batch": w.batch, "layers": w.layers, "heads": w.heads, "head_dim": w.head_dim,
+            "prompt_len": w.prompt_len, "keep_ratio": w.keep_ratio, "decode_steps": w.decode_steps,
+            "offset": w.offset, "population": "per_head", "protect_ends": True,
+            "l2": "inputs larger than L2 (prompt Q/K/V and the compacted cache each exceed 126 MB per pass)"}
+
+
+# ----------------------------------------------------------------------------- GPU leg
+
+def run_ours(args, w: wl.Workload):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2407_18121_b200 import binding as ec
+    from paper_2407_18121_b200 import build as ecbuild
+    from paper_2407_18121_b200.session import ElasticCacheSession
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        ecbuild.build()
+    if world > 1:
+        dist.barrier()
+    ec.lib()
+
+    # every rank holds its own batch of independent problems (weak scaling, no exchange)
+    import dataclasses
+    wr = dataclasses.replace(w, seed=w.seed + 1000 * rank)
+    N, H, T, D, S = wr.N, wr.heads, wr.prompt_len, wr.head_dim, wr.decode_steps
+    Qb, Kb, Vb = wl.prompt(wr)
+    qb, kb, vb = wl.decode_inputs(wr)
+    Qh, Kh, Vh = (bits_to_tensor(x, True) for x in (Qb, Kb, Vb))
+    qh, kh, vh = (bits_to_tensor(x, True) for x in (qb, kb, vb))
+    Q, K, V = Qh.cuda(), Kh.cuda(), Vh.cuda()
+    q, k, v = qh.cuda(), kh.cuda(), vh.cuda()
+    out = torch.empty_like(q)
+    out_h = torch.empty(q.shape, dtype=torch.bfloat16).pin_memory()
+    anchors_h = torch.empty((N, H, ec.ec_keep_count(T, wr.keep_ratio)), dtype=torch.int32).pin_memory()
+
+    sess = ElasticCacheSession(N, H, T, D, wr.keep_ratio, wr.offset, wr.scale)
+    C = sess.n_keep
+    units = N * H
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def one_pass(events=None):
+        if events is not None:
+            events[0].record(stream)
+        ec.ec_importance(Q, K, sess.scores, None, sess.scale, sess.ws_imp)
+        if events is not None:
+            events[1].record(stream)
+        ec.ec_select_merge(K, V, sess.scores, C, sess.population, True, sess.Kc, sess.Vc, sess.anchor_pos,
+                           None, sess.ws_sel)
+        sess.cache = ec.ec_cache_init(sess.Kc, sess.Vc, C, C, wr.offset)
+        if events is not None:
+            events[2].record(stream)
+        sess.decode(q, k, v, out)
+        if events is not None:
+            events[3].record(stream)
+
+    for _ in range(args.warmup):
+        one_pass()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record(stream)
+    for i in range(args.steps):
+        one_pass(ev[i])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    imp_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    mrg_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    dec_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
+    status = ec.ec_device_status(sess.ws_imp)
+    if status != ec.EC_OK:
+        raise SystemExit(f"device status {status}: {ec.status_string(status)}")
+
+    # end to end: inputs start in pinned host memory, results are read back every pass
+    for _ in range(max(1, min(args.warmup, 2))):
+        sess.compress_host(Qh, Kh, Vh, anchors_h)
+        sess.decode_host(qh, kh, vh, out_h)
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(1, min(args.steps, 3))
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        h2d_a = sess.compress_host(Qh, Kh, Vh, anchors_h)
+        h2d_b, d2h_b = sess.decode_host(qh, kh, vh, out_h)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    h2d = h2d_a + h2d_b
+    d2h = d2h_b + anchors_h.numel() * 4
+
+    ms_per_step = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    tokens = w.batch * S * world
+    value = tokens / (ms_per_step * 1e-3)
+    # algorithmic bytes of one decode launch: every cached K and V row once, q/k_new/v_new in,
+    # out and the overwritten slot (K and V row) out
+    dec_bytes = units * (2 * C * D * 2 + 3 * D * 2 + D * 2 + 2 * D * 2)
+    dec_launch_s = dec_ms * 1e-3 / S
+    dec_gbs = dec_bytes / dec_launch_s / 1e9
+    mrg_bytes = units * (2 * T * D * 2 + 4 * T + 2 * C * D * 2 + 4 * C)
+    mrg_gbs = mrg_bytes / (mrg_ms * 1e-3) / 1e9
+    imp_flops = 2.0 * D * T * (T + 1) * units   # two passes, each 2*D flops for T(T+1)/2 causal scores
+    imp_tflops = imp_flops / (imp_ms * 1e-3) / 1e12
+    splits = 1 if units >= 592 else None
+    launches_per_pass = 2 + 2 + S * (1 if splits == 1 else 2)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 storage, fp32 arithmetic", "data": "synthetic",
+        "config": workload_config(w),
+        "stages_ms": {"importance": imp_ms, "select_merge": mrg_ms, "decode_loop": dec_ms,
+                      "decode_per_token_us": dec_ms * 1e3 / S},
+        "decode_only_tokens_per_s": w.batch * S * world / (dec_ms * 1e-3),
+        "roofline": {"kernel": "decode_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     "frac_of_nominal_8TBs": dec_gbs / 8000.0, "bytes_per_launch": dec_bytes, "traffic": None},
+        "merge": {"achieved": mrg_gbs, "unit": "GB/s", "frac": mrg_gbs / peaks["hbm_gbs"],
+                  "frac_of_nominal_8TBs": mrg_gbs / 8000.0, "bytes_per_call": mrg_bytes,
+                  "note": "whole ec_select_merge call (selection + merge kernels)"},
+        "importance": {"achieved": imp_tflops, "unit": "TFLOP/s", "frac": imp_tflops / peaks["bf16_tflops"],
+                       "flops_per_call": imp_flops},
+        "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_pass * args.steps,
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        o = oracle_sample(w, args.oracle_decode_steps, args.oracle_problems)
+        line["cpu_baseline"] = {"value": w.batch * S / o["seconds_whole_pass_extrapolated"], "unit": UNIT,
+                                "cores": o["cores"], "kind": "oracle", "sample": o["sample"],
+                                "sample_seconds": o["sample_seconds"]}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llava7b_b1", choices=list(wl.WORKLOADS))
+    ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode length")
+    ap.add_argument("--oracle-decode-steps", type=int, default=64)
+    ap.add_argument("--oracle-problems", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = wl.WORKLOADS[args.workload]
+    if args.decode_steps:
+        w = w.shrunk(decode_steps=args.decode_steps)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,98 @@
+"""Buffer management around the C ABI: owns the device tensors and workspaces of one
+workload shape and sequences the three calls. No arithmetic happens here.
+
+    s = ElasticCacheSession(N, H, T, D, keep_ratio=0.5, offset=16, scale=1/sqrt(D))
+    s.compress(Q, K, V)                  # importance -> select/merge; cache ready, len = budget
+    s.decode(q_all, k_all, v_all, out)   # [steps, N, H, D] each; fixed-point eviction every step
+
+`compress_host` / `decode_host` take pinned host tensors and include the host<->device
+copies (on the current stream), for callers whose data starts on the host.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as ec
+
+
+class ElasticCacheSession:
+    def __init__(self, N: int, H: int, T: int, D: int, keep_ratio: float, offset: int, scale: float,
+                 population: int = ec.EC_PER_HEAD, protect_ends: bool = True, extra_rows: int = 0,
+                 device: Optional[torch.device] = None):
+        self.N, self.H, self.T, self.D = N, H, T, D
+        self.scale = float(scale)
+        self.offset = int(offset)
+        self.population = population
+        self.protect_ends = protect_ends
+        self.n_keep = ec.ec_keep_count(T, keep_ratio)
+        if self.n_keep < 1:
+            raise ValueError("invalid prompt length or keep ratio")
+        self.cap = self.n_keep + extra_rows
+        dev = device or torch.device("cuda", torch.cuda.current_device())
+        self.device = dev
+        bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
+        self.scores = torch.empty((N, H, T), dtype=f32, device=dev)
+        self.Kc = torch.empty((N, H, self.cap, D), dtype=bf, device=dev)
+        self.Vc = torch.empty_like(self.Kc)
+        self.anchor_pos = torch.empty((N, H, self.n_keep), dtype=i32, device=dev)
+        self.ws_imp = torch.empty(ec.ec_importance_workspace(N, H, T, D), dtype=torch.uint8, device=dev)
+        self.ws_sel = torch.empty(ec.ec_select_merge_workspace(N, H, T, D, self.n_keep, population),
+                                  dtype=torch.uint8, device=dev)
+        self.cache = ec.ec_cache_init(self.Kc, self.Vc, 0, max(self.n_keep, 2), min(self.offset, max(self.n_keep, 2) - 1))
+        self.ws_dec = torch.empty(ec.ec_decode_workspace(self.cache), dtype=torch.uint8, device=dev)
+        self._stage = None      # device staging for the *_host calls, allocated on first use
+        self._dstage = None
+
+    # ---- device-resident inputs ------------------------------------------------------
+    def compress(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor) -> None:
+        """Prompt call: importance, anchor selection and merge. Resets the cache to `n_keep` rows."""
+        ec.ec_importance(Q, K, self.scores, None, self.scale, self.ws_imp)
+        ec.ec_select_merge(K, V, self.scores, self.n_keep, self.population, self.protect_ends,
+                           self.Kc, self.Vc, self.anchor_pos, None, self.ws_sel)
+        self.cache = ec.ec_cache_init(self.Kc, self.Vc, self.n_keep, max(self.n_keep, 2),
+                                      min(self.offset, max(self.n_keep, 2) - 1))
+
+    def decode(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, out: torch.Tensor,
+               want_slots: bool = False):
+        """Generation calls for q, k_new, v_new, out of shape [steps, N, H, D]."""
+        return ec.ec_decode_steps(q, k_new, v_new, self.cache, self.scale, out, self.ws_dec, want_slots)
+
+    # ---- host-resident inputs --------------------------------------------------------
+    def _prompt_staging(self):
+        if self._stage is None:
+            shp = (self.N, self.H, self.T, self.D)
+            self._stage = tuple(torch.empty(shp, dtype=torch.bfloat16, device=self.device) for _ in range(3))
+        return self._stage
+
+    def _decode_staging(self, steps: int):
+        if self._dstage is None or self._dstage[0].shape[0] < steps:
+            shp = (steps, self.N, self.H, self.D)
+            self._dstage = tuple(torch.empty(shp, dtype=torch.bfloat16, device=self.device) for _ in range(4))
+        return self._dstage
+
+    def compress_host(self, Q_host: torch.Tensor, K_host: torch.Tensor, V_host: torch.Tensor,
+                      anchor_pos_host: Optional[torch.Tensor] = None) -> int:
+        """compress() from pinned host tensors. Returns the bytes copied host->device."""
+        Q, K, V = self._prompt_staging()
+        Q.copy_(Q_host, non_blocking=True)
+        K.copy_(K_host, non_blocking=True)
+        V.copy_(V_host, non_blocking=True)
+        self.compress(Q, K, V)
+        if anchor_pos_host is not None:
+            anchor_pos_host.copy_(self.anchor_pos, non_blocking=True)
+        return 3 * Q_host.numel() * Q_host.element_size()
+
+    def decode_host(self, q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor,
+                    out_host: torch.Tensor):
+        """decode() from pinned host tensors [steps, N, H, D]; writes out_host. Returns (h2d, d2h) bytes."""
+        steps = q_host.shape[0]
+        q, k, v, out = (t[:steps] for t in self._decode_staging(steps))
+        q.copy_(q_host, non_blocking=True)
+        k.copy_(k_host, non_blocking=True)
+        v.copy_(v_host, non_blocking=True)
+        self.decode(q, k, v, out)
+        out_host.copy_(out, non_blocking=True)
+        nb = q_host.numel() * q_host.element_size()
+        return 3 * nb, nb
