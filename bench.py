@@ -105,12 +105,25 @@ def bits_to_tensor(bits: np.ndarray, pin: bool):
 
 # ----------------------------------------------------------------------------- CPU oracle leg
 
-def oracle_sample(w: wl.Workload, decode_steps_sample: int, problems_sample: int):
-    """Times the oracle on a bounded sample and extrapolates to the whole pass.
+def oracle_sample_size(w: wl.Workload, budget_fma: float = 2.0e11):
+    """Picks how much of the workload the oracle is timed on: the whole pass when its
+    multiply-add count fits the budget (tens of seconds on a many-core host), otherwise the
+    first problems and the first decode steps, in proportion."""
+    C_keep = w.prompt_len - int(w.prompt_len - w.prompt_len * w.keep_ratio)
+    prompt = w.heads * w.prompt_len * (w.prompt_len + 1) / 2 * w.head_dim          # per problem
+    decode = w.heads * (C_keep + 1) * w.head_dim * 2                              # per problem per step
+    problems = int(max(1, min(w.N, (budget_fma / 2) // prompt)))
+    steps = int(max(4, min(w.decode_steps, (budget_fma / 2) // (decode * problems))))
+    return problems, steps
+
+
+def oracle_sample(w: wl.Workload, decode_steps_sample: int = 0, problems_sample: int = 0):
+    """Times the oracle, as it stands, on a bounded sample and scales linearly to the whole pass.
     Sample: the full prompt stage (importance, selection, buckets, merge) of the first
     `problems_sample` problems, then `decode_steps_sample` decode steps on them."""
     from oracle import ec_oracle as orc
-    problems = list(range(min(problems_sample, w.N)))
+    auto_p, auto_s = oracle_sample_size(w)
+    problems = list(range(min(problems_sample or auto_p, w.N)))
     Qb, Kb, Vb = wl.prompt(w, problems)
     T = w.prompt_len
     C = orc.keep_count(T, w.keep_ratio)
@@ -121,7 +134,7 @@ def oracle_sample(w: wl.Workload, decode_steps_sample: int, problems_sample: int
     Kc, Vc = orc.merge(Kb, lo, hi), orc.merge(Vb, lo, hi)
     queue = orc.DecodeQueue(orc.widen_bf16(orc.round_bf16(Kc)), orc.widen_bf16(orc.round_bf16(Vc)), cap=C + 1)
     t1 = time.perf_counter()
-    S = min(decode_steps_sample, w.decode_steps)
+    S = min(decode_steps_sample or auto_s, w.decode_steps)
     dec_in = [wl.decode_step_inputs(w, s, problems) for s in range(S)]
     t2 = time.perf_counter()
     for s in range(S):
@@ -132,10 +145,12 @@ def oracle_sample(w: wl.Workload, decode_steps_sample: int, problems_sample: int
     prompt_s = (t1 - t0) * frac
     decode_s = (t3 - t2) * frac * (w.decode_steps / S)
     total = prompt_s + decode_s
+    whole = len(problems) == w.N and S == w.decode_steps
     return {"seconds_whole_pass_extrapolated": total, "prompt_s": prompt_s, "decode_s": decode_s,
             "sample_seconds": (t1 - t0) + (t3 - t2), "cores": orc.num_threads(),
-            "sample": (f"prompt stage of {len(problems)} of {w.N} problems (all {w.heads} heads) + {S} of "
-                       f"{w.decode_steps} decode steps on them, extrapolated linearly to the whole pass")}
+            "sample": ("the whole pass (every problem, every decode step)" if whole else
+                       f"prompt stage of {len(problems)} of {w.N} problems (all {w.heads} heads) + {S} of "
+                       f"{w.decode_steps} decode steps on them, scaled linearly to the whole pass")}
 
 
 def run_reference(args, w: wl.Workload):
@@ -340,8 +355,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llava7b_b1", choices=list(wl.WORKLOADS))
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode length")
-    ap.add_argument("--oracle-decode-steps", type=int, default=64)
-    ap.add_argument("--oracle-problems", type=int, default=16)
+    ap.add_argument("--oracle-decode-steps", type=int, default=0)
+    ap.add_argument("--oracle-problems", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = wl.WORKLOADS[args.workload]
