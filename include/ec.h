@@ -46,7 +46,8 @@ typedef enum {
     EC_ERR_ARG = 4,       /* a scalar argument is out of range                           */
     EC_ERR_WORKSPACE = 5, /* workspace missing or smaller than the query reports         */
     EC_ERR_CUDA = 6,      /* a CUDA runtime call failed (launch error, no device, ...)   */
-    EC_ERR_TIMEOUT = 7    /* a bounded device-side wait expired (see ec_device_status)   */
+    EC_ERR_TIMEOUT = 7,   /* a bounded device-side wait expired (see ec_device_status)   */
+    EC_ERR_TOO_LARGE = 8  /* the problem does not fit the library's built-in scratch      */
 } ec_status;
 
 /* Static description of a status code; never NULL. */
@@ -178,6 +179,33 @@ int ec_decode_step(const void *q_dev, const void *k_new_dev, const void *v_new_d
 int ec_decode_steps(const void *q_dev, const void *k_new_dev, const void *v_new_dev, int steps,
                     ec_cache *c, float scale, void *out_dev, int *evicted_slots_host,
                     void *ws_dev, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------- no-allocation decode */
+
+/*
+ * (No counterpart in the paper: this is a deployment convenience.)
+ *
+ * ec_decode_step for callers that cannot allocate device memory and therefore cannot
+ * provide the workspace: a server whose memory pool took the whole GPU at start-up, a
+ * plug-in whose execute hook must not call cudaMalloc, a latency-critical loop that cannot
+ * take cudaMalloc's device-wide synchronisation. Arguments, results and state updates are
+ * those of ec_decode_step without ws/ws_bytes; the scratch is a fixed array inside the
+ * library of ec_decode_noalloc_capacity() bytes (2 MiB, resident on every GPU that loads
+ * the library until the process exits). The call itself allocates and frees nothing.
+ *
+ *  - Limit: ec_decode_workspace(c) must not exceed the capacity (at D = 128 about 4000
+ *    units, N*H); otherwise EC_ERR_TOO_LARGE is returned and nothing is launched.
+ *  - The first call on each device looks up the array's device address (a one-time runtime
+ *    query, made with that device current). Make that first call outside any stream capture.
+ *  - All calls on a device share the one array, which keeps whatever the previous call left
+ *    there. Each launch rewrites the part it reads, so no clearing is needed, but two calls
+ *    whose kernels may run at the same time (different streams, different caches) race on
+ *    it: serialise them.
+ */
+size_t ec_decode_noalloc_capacity(void);
+int ec_decode_step_noalloc(const void *q_dev, const void *k_new_dev, const void *v_new_dev,
+                           ec_cache *c, float scale, void *out_dev,
+                           int *evicted_slot_host, int *slot_written_host, void *stream);
 
 #ifdef __cplusplus
 }

@@ -25,6 +25,7 @@ EXPORTS = (
     "ec_importance_workspace", "ec_importance", "ec_device_status",
     "ec_select_merge_workspace", "ec_select_merge",
     "ec_cache_init", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
+    "ec_decode_noalloc_capacity", "ec_decode_step_noalloc",
 )
 
 
@@ -77,6 +78,10 @@ def lib() -> C.CDLL:
     L.ec_decode_step.argtypes = [vp, vp, vp, C.POINTER(ec_cache), f, vp, C.POINTER(i), C.POINTER(i), vp, sz, vp]
     L.ec_decode_steps.restype = i
     L.ec_decode_steps.argtypes = [vp, vp, vp, i, C.POINTER(ec_cache), f, vp, C.POINTER(i), vp, sz, vp]
+    L.ec_decode_noalloc_capacity.restype = sz
+    L.ec_decode_noalloc_capacity.argtypes = []
+    L.ec_decode_step_noalloc.restype = i
+    L.ec_decode_step_noalloc.argtypes = [vp, vp, vp, C.POINTER(ec_cache), f, vp, C.POINTER(i), C.POINTER(i), vp]
     _lib = L
     return L
 
@@ -175,3 +180,20 @@ def ec_decode_steps(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, c
                                slots, _ptr(ws), ws.numel() * ws.element_size(), _stream())
     _check(st, "ec_decode_steps")
     return list(slots) if want_slots else None
+
+
+def ec_decode_noalloc_capacity() -> int:
+    return int(lib().ec_decode_noalloc_capacity())
+
+
+def ec_decode_step_noalloc(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, cache: ec_cache,
+                           scale: float, out: torch.Tensor):
+    """ec_decode_step without a workspace argument, for callers that may not allocate device
+    memory: the scratch is a fixed 2 MiB array inside the library. Raises EcError with status
+    EC_ERR_TOO_LARGE when the cache is too big for it. Calls that could overlap on the GPU must
+    be serialised by the caller, since they share that array."""
+    ev, sl = C.c_int(-1), C.c_int(-1)
+    st = lib().ec_decode_step_noalloc(_ptr(q), _ptr(k_new), _ptr(v_new), C.byref(cache), float(scale), _ptr(out),
+                                      C.byref(ev), C.byref(sl), _stream())
+    _check(st, "ec_decode_step_noalloc")
+    return ev.value, sl.value

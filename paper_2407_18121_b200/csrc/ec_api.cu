@@ -36,6 +36,7 @@ const char *ec_status_string(int status)
     case EC_ERR_WORKSPACE: return "workspace missing or too small";
     case EC_ERR_CUDA: return "CUDA runtime error";
     case EC_ERR_TIMEOUT: return "device-side wait timed out";
+    case EC_ERR_TOO_LARGE: return "problem too large for the built-in scratch";
     default: return "unknown status";
     }
 }
