@@ -110,7 +110,7 @@ size_t ec_select_merge_workspace(int N, int H, int T, int D, int n_keep, int pop
  *  2. bucket k = positions floor((t_{k-1}+t_k)/2)+1 .. floor((t_k+t_{k+1})/2), the first
  *     bucket starting at 0 and the last ending at T-1.
  *  3. row k of the compacted cache = arithmetic mean of the bucket's rows (fp32
- *     accumulation in position order, one rounding to bf16), for K and for V.
+ *     accumulation in position order, scaled by 1/size, one rounding to bf16), for K and for V.
  *
  *   K_dev, V_dev    bf16 [N, H, T, D]                                     (in)
  *   scores_dev      fp32 [N, H, T]                                        (in)

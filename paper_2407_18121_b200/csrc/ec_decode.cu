@@ -7,8 +7,20 @@ namespace ec {
 
 namespace {
 
-constexpr int kDecThreads = 256;
-constexpr int kRowsPerIter = 4;
+// Tunables (compile-time): threads per CTA and cache rows a lane group fetches per iteration.
+// 128-thread CTAs keep at least 7 CTAs resident per SM, so that the 1024 units of a 7B-shaped
+// single-sequence step (6.9 per SM) all run in one balanced wave.
+#ifndef EC_DEC_THREADS
+#define EC_DEC_THREADS 128
+#endif
+#ifndef EC_DEC_ROWS
+#define EC_DEC_ROWS 4
+#endif
+#ifndef EC_DEC_MIN_CTAS
+#define EC_DEC_MIN_CTAS 7
+#endif
+constexpr int kDecThreads = EC_DEC_THREADS;
+constexpr int kRowsPerIter = EC_DEC_ROWS;
 
 // The cache is written later in the same kernel, so no read-only (.nc) path here.
 __device__ __forceinline__ uint4 ld_row(const uint4 *p)
@@ -25,7 +37,7 @@ __device__ __forceinline__ uint4 ld_row(const uint4 *p)
 // splits == 1: writes out (bf16) and stores the new row into `write_slot`.
 // splits  > 1: writes (acc[D], max, sum) per split to `partials`; the combine kernel finishes.
 template <int LPR>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, EC_DEC_MIN_CTAS)
 decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
               uint4 *Kc, uint4 *Vc, int cap, int len, int write_slot, float scale_log2e,
               __nv_bfloat16 *__restrict__ out, float *__restrict__ partials, int splits)
@@ -110,8 +122,7 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
     for (int i = 0; i < 8; ++i) sm_acc[g][l * 8 + i] = acc[i];
     __syncthreads();   // also orders every cache read of this CTA before the slot write below
 
-    if (threadIdx.x < D) {
-        const int d = threadIdx.x;
+    for (int d = threadIdx.x; d < D; d += kDecThreads) {
         float M = -INFINITY;
 #pragma unroll
         for (int gg = 0; gg < G; ++gg) M = fmaxf(M, sm_m[gg]);

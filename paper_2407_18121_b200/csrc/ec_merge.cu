@@ -1,73 +1,116 @@
 // Bucket division (Eq. 2) and mean merge (Eq. 3) into the dense compacted cache.
 // HBM-bound streaming: every prompt row of K and V is read exactly once with 16-byte loads,
 // every kept row is written once.
+//
+// Buckets are consecutive row ranges, so a run of buckets is one contiguous range of prompt
+// rows. A CTA takes a slice of prompt rows of one unit; each lane group takes an equal part
+// of the slice, owns the buckets that START inside its part, and streams their rows in order
+// (addresses do not depend on the bucket structure, so many loads are in flight), flushing a
+// mean whenever it passes a bucket's last row.
 #include "ec_common.cuh"
 
 namespace ec {
 
 namespace {
 
-constexpr int kMergeThreads = 256;
-constexpr int kRowsPerCta = 64;   // output rows (buckets) handled by one CTA
+#ifndef EC_MERGE_THREADS
+#define EC_MERGE_THREADS 128
+#endif
+#ifndef EC_MERGE_ROWS_PER_CTA
+#define EC_MERGE_ROWS_PER_CTA 256
+#endif
+#ifndef EC_MERGE_UNROLL
+#define EC_MERGE_UNROLL 4
+#endif
+constexpr int kMergeThreads = EC_MERGE_THREADS;
+constexpr int kRowsPerCta = EC_MERGE_ROWS_PER_CTA;
+constexpr int kUnroll = EC_MERGE_UNROLL;
+
+// First row of bucket k (Eq. 2): one past the midpoint between anchors k-1 and k.
+__device__ __forceinline__ int bucket_lo(const int32_t *anch, int k)
+{
+    return (k == 0) ? 0 : ((anch[k - 1] + anch[k]) >> 1) + 1;
+}
+
+// Smallest k in [0, C] whose bucket starts at or after row r (C when none does).
+__device__ __forceinline__ int first_bucket_from(const int32_t *anch, int C, int r)
+{
+    int lo = 0, hi = C;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (bucket_lo(anch, mid) >= r) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
 
 // LPR = lanes per row = D / 8 (each lane holds 8 bf16 = 16 bytes of a row).
-// grid.x = units * chunks; a lane group walks buckets k0+g, k0+g+G, ... of its chunk and
-// sums the bucket's rows in position order in fp32.
+// grid.x = units * slices. Dynamic shared memory: the unit's C anchors.
 template <int LPR>
 __global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int32_t *__restrict__ anchor_pos,
-             int T, int C, int chunks, uint4 *__restrict__ Kc, uint4 *__restrict__ Vc, int cap)
+             int T, int C, int slices, uint4 *__restrict__ Kc, uint4 *__restrict__ Vc, int cap)
 {
     constexpr int G = kMergeThreads / LPR;          // lane groups per CTA
-    const int unit = blockIdx.x / chunks;
-    const int chunk = blockIdx.x - unit * chunks;
+    extern __shared__ int32_t anch[];
+    const int unit = blockIdx.x / slices;
+    const int slice = blockIdx.x - unit * slices;
     const int g = threadIdx.x / LPR;
     const int l = threadIdx.x - g * LPR;
-    const int32_t *anch = anchor_pos + (size_t)unit * C;
-    const uint4 *Ku = K + (size_t)unit * T * LPR;
-    const uint4 *Vu = V + (size_t)unit * T * LPR;
-    uint4 *Kcu = Kc + (size_t)unit * cap * LPR;
-    uint4 *Vcu = Vc + (size_t)unit * cap * LPR;
 
-    const int k_end = min((chunk + 1) * kRowsPerCta, C);
-    for (int k = chunk * kRowsPerCta + g; k < k_end; k += G) {
-        const int a = anch[k];
-        const int lo = (k == 0) ? 0 : ((anch[k - 1] + a) >> 1) + 1;
-        const int hi = (k == C - 1) ? T - 1 : ((a + anch[k + 1]) >> 1);
-        float ak[8], av[8];
+    const int32_t *ap = anchor_pos + (size_t)unit * C;
+    for (int k = threadIdx.x; k < C; k += kMergeThreads) anch[k] = ap[k];
+    __syncthreads();
+
+    const int R0 = slice * kRowsPerCta, R1 = min(R0 + kRowsPerCta, T);
+    const int part = (R1 - R0 + G - 1) / G;
+    const int ra = min(R0 + g * part, R1), rb = min(ra + part, R1);
+    int k = first_bucket_from(anch, C, ra);
+    const int k_end = first_bucket_from(anch, C, rb);
+    if (k >= k_end) return;
+
+    const uint4 *Ku = K + (size_t)unit * T * LPR + l;
+    const uint4 *Vu = V + (size_t)unit * T * LPR + l;
+    uint4 *Kcu = Kc + (size_t)unit * cap * LPR + l;
+    uint4 *Vcu = Vc + (size_t)unit * cap * LPR + l;
+
+    int lo = bucket_lo(anch, k);
+    const int last = (k_end == C) ? T - 1 : bucket_lo(anch, k_end) - 1;   // last row this group reads
+    int hi = (k == C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
+    float ak[8], av[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { ak[i] = 0.f; av[i] = 0.f; }
-        int t = lo;
-        for (; t + 3 <= hi; t += 4) {
-            uint4 rk[4], rv[4];
+    for (int i = 0; i < 8; ++i) { ak[i] = 0.f; av[i] = 0.f; }
+
+    for (int t = lo; t <= last; t += kUnroll) {
+        uint4 rk[kUnroll], rv[kUnroll];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                rk[j] = ldg_stream(Ku + (size_t)(t + j) * LPR + l);
-                rv[j] = ldg_stream(Vu + (size_t)(t + j) * LPR + l);
+        for (int j = 0; j < kUnroll; ++j) {
+            if (t + j <= last) {
+                rk[j] = ldg_stream(Ku + (size_t)(t + j) * LPR);
+                rv[j] = ldg_stream(Vu + (size_t)(t + j) * LPR);
             }
+        }
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kUnroll; ++j) {
+            if (t + j <= last) {
                 float fk[8], fv[8];
                 unpack8(rk[j], fk);
                 unpack8(rv[j], fv);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) { ak[i] += fk[i]; av[i] += fv[i]; }
+                if (t + j == hi) {
+                    const float inv = 1.0f / (float)(hi - lo + 1);      // exactly 1 for a singleton bucket
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { ak[i] *= inv; av[i] *= inv; }
+                    Kcu[(size_t)k * LPR] = pack8(ak);
+                    Vcu[(size_t)k * LPR] = pack8(av);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { ak[i] = 0.f; av[i] = 0.f; }
+                    ++k;
+                    lo = hi + 1;
+                    hi = (k >= C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
+                }
             }
         }
-        for (; t <= hi; ++t) {
-            uint4 rk = ldg_stream(Ku + (size_t)t * LPR + l);
-            uint4 rv = ldg_stream(Vu + (size_t)t * LPR + l);
-            float fk[8], fv[8];
-            unpack8(rk, fk);
-            unpack8(rv, fv);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { ak[i] += fk[i]; av[i] += fv[i]; }
-        }
-        const float cnt = (float)(hi - lo + 1);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { ak[i] = ak[i] / cnt; av[i] = av[i] / cnt; }
-        Kcu[(size_t)k * LPR + l] = pack8(ak);
-        Vcu[(size_t)k * LPR + l] = pack8(av);
     }
 }
 
@@ -76,15 +119,24 @@ merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int
 cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
                          int n_keep, void *Kc, void *Vc, int cap, cudaStream_t stream)
 {
-    const int chunks = (n_keep + kRowsPerCta - 1) / kRowsPerCta;
-    const long long grid = (long long)units * chunks;
+    const int slices = (T + kRowsPerCta - 1) / kRowsPerCta;
+    const long long grid = (long long)units * slices;
     if (grid > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    const size_t smem = (size_t)n_keep * sizeof(int32_t);
     if (D == 128) {
-        merge_kernel<16><<<(unsigned)grid, kMergeThreads, 0, stream>>>(
-            (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, chunks, (uint4 *)Kc, (uint4 *)Vc, cap);
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(merge_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        merge_kernel<16><<<(unsigned)grid, kMergeThreads, smem, stream>>>(
+            (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, slices, (uint4 *)Kc, (uint4 *)Vc, cap);
     } else {
-        merge_kernel<8><<<(unsigned)grid, kMergeThreads, 0, stream>>>(
-            (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, chunks, (uint4 *)Kc, (uint4 *)Vc, cap);
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(merge_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        merge_kernel<8><<<(unsigned)grid, kMergeThreads, smem, stream>>>(
+            (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, slices, (uint4 *)Kc, (uint4 *)Vc, cap);
     }
     return cudaGetLastError();
 }
