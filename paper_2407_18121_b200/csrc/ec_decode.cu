@@ -1,26 +1,29 @@
 // Decode attention over the compacted cache plus the step's new row, with the new row
 // written into the slot freed by fixed-point elimination (Sec. 3.3 "Output Generation").
-// HBM-bound: every cached K and V row is read once per step with 16-byte loads.
+// HBM-bound: every cached K and V row is read once per step with 16-byte loads, so the
+// kernel is built to spend as few instructions per byte as possible:
+//  - LPR = D/8 lanes share a row (8 bf16 each); a lane group takes blocks of 8 consecutive
+//    rows, so 16 independent 16-byte loads per lane are in flight;
+//  - the 8 partial dot products of a block are reduced across the group with a transposing
+//    butterfly (7 shuffles instead of 8 x log2(LPR)), which leaves each row's score on one lane
+//    (pair), so the exponential is evaluated once per row, not once per lane;
+//  - multiply-adds are issued as packed fp32 pairs (__ffma2_rn).
 #include "ec_common.cuh"
 
 namespace ec {
 
 namespace {
 
-// Tunables (compile-time): threads per CTA and cache rows a lane group fetches per iteration.
-// 128-thread CTAs keep at least 7 CTAs resident per SM, so that the 1024 units of a 7B-shaped
-// single-sequence step (6.9 per SM) all run in one balanced wave.
+// Threads per CTA. Small CTAs let at least 7 be resident per SM, so that the 1024 units of a
+// 7B-shaped single-sequence step (6.9 per SM) run as one balanced wave.
 #ifndef EC_DEC_THREADS
-#define EC_DEC_THREADS 128
-#endif
-#ifndef EC_DEC_ROWS
-#define EC_DEC_ROWS 4
+#define EC_DEC_THREADS 64
 #endif
 #ifndef EC_DEC_MIN_CTAS
-#define EC_DEC_MIN_CTAS 7
+#define EC_DEC_MIN_CTAS 8
 #endif
 constexpr int kDecThreads = EC_DEC_THREADS;
-constexpr int kRowsPerIter = EC_DEC_ROWS;
+constexpr int kBlk = 8;                       // rows per block of a lane group
 
 // The cache is written later in the same kernel, so no read-only (.nc) path here.
 __device__ __forceinline__ uint4 ld_row(const uint4 *p)
@@ -31,9 +34,96 @@ __device__ __forceinline__ uint4 ld_row(const uint4 *p)
     return v;
 }
 
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+__device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16lo(w), bf16hi(w)); }
+
+// Partial dot product of this lane's 8 elements (q pre-multiplied by scale*log2e).
+__device__ __forceinline__ float dot8(const float2 (&q2)[4], const uint4 &k)
+{
+    float2 d = __ffma2_rn(q2[0], unpack2(k.x), make_float2(0.f, 0.f));
+    d = __ffma2_rn(q2[1], unpack2(k.y), d);
+    d = __ffma2_rn(q2[2], unpack2(k.z), d);
+    d = __ffma2_rn(q2[3], unpack2(k.w), d);
+    return d.x + d.y;
+}
+
+__device__ __forceinline__ void axpy8(float2 (&acc)[4], float p, const uint4 &v)
+{
+    const float2 p2 = make_float2(p, p);
+    acc[0] = __ffma2_rn(p2, unpack2(v.x), acc[0]);
+    acc[1] = __ffma2_rn(p2, unpack2(v.y), acc[1]);
+    acc[2] = __ffma2_rn(p2, unpack2(v.z), acc[2]);
+    acc[3] = __ffma2_rn(p2, unpack2(v.w), acc[3]);
+}
+
+// Running softmax state of a lane group, log2 domain. `lsum` is a per-lane partial: each
+// row's weight is added on the lanes that own the row (LPR/8 of them).
+struct GroupState {
+    float m, lsum;
+    float2 acc[4];
+};
+
+// One block of up to 8 consecutive cache rows starting at `row`. GUARD: rows >= row_end are
+// skipped (their loads are clamped to the last valid row and their score is -inf).
+template <int LPR, bool GUARD>
+__device__ __forceinline__ void process_block(GroupState &st, const float2 (&q2)[4], const uint4 *Kl, const uint4 *Vl,
+                                              int row, int row_end, int l, unsigned gmask)
+{
+    uint4 rk[kBlk], rv[kBlk];
+#pragma unroll
+    for (int r = 0; r < kBlk; ++r) {
+        const int j = GUARD ? min(row + r, row_end - 1) : row + r;
+        rk[r] = ld_row(Kl + (size_t)j * LPR);
+    }
+#pragma unroll
+    for (int r = 0; r < kBlk; ++r) {
+        const int j = GUARD ? min(row + r, row_end - 1) : row + r;
+        rv[r] = ld_row(Vl + (size_t)j * LPR);
+    }
+    float s[kBlk];
+#pragma unroll
+    for (int r = 0; r < kBlk; ++r) s[r] = dot8(q2, rk[r]);
+
+    // transposing butterfly: after the three steps lane l holds the sum for row (l * 8 / LPR)
+#pragma unroll
+    for (int step = 0; step < 3; ++step) {
+        const int o = LPR >> (step + 1);
+        const int n = kBlk >> step;                 // values held before this step
+        const bool upper = (l & o) != 0;
+#pragma unroll
+        for (int i = 0; i < n / 2; ++i) {
+            const float keep = upper ? s[i + n / 2] : s[i];
+            const float send = upper ? s[i] : s[i + n / 2];
+            s[i] = keep + __shfl_xor_sync(gmask, send, o);
+        }
+    }
+    float sc = s[0];
+    if (LPR == 16) sc += __shfl_xor_sync(gmask, sc, 1);
+    if (GUARD) {
+        const int my_row = row + l * kBlk / LPR;
+        if (my_row >= row_end) sc = -INFINITY;
+    }
+    float bm = sc;
+#pragma unroll
+    for (int o = LPR / 2; o >= LPR / 8; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(gmask, bm, o));
+    const float mn = fmaxf(st.m, bm);               // finite: a block always has a valid first row
+    const float corr = fast_exp2(st.m - mn);        // first block: exp2(-inf) = 0
+    const float p = fast_exp2(sc - mn);
+    st.m = mn;
+    st.lsum = fmaf(st.lsum, corr, p);
+    const float2 c2 = make_float2(corr, corr), z2 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) st.acc[i] = __ffma2_rn(st.acc[i], c2, z2);
+#pragma unroll
+    for (int r = 0; r < kBlk; ++r) {
+        const float pr = __shfl_sync(gmask, p, r * LPR / kBlk, LPR);
+        axpy8(st.acc, pr, rv[r]);
+    }
+}
+
 // grid.x = units * splits. Rows 0..len-1 come from the cache, row `len` is the new token.
-// LPR lanes share one row (8 bf16 each); a lane group keeps a running (max, sum, acc) in
-// the log2 domain and the CTA merges its groups through shared memory.
 // splits == 1: writes out (bf16) and stores the new row into `write_slot`.
 // splits  > 1: writes (acc[D], max, sum) per split to `partials`; the combine kernel finishes.
 template <int LPR>
@@ -47,6 +137,12 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
     __shared__ float sm_acc[G][D];
     __shared__ float sm_m[G], sm_l[G];
 
+    // Launched with programmatic stream serialization: nothing in global memory is touched
+    // before the previous kernel of the stream has completed; the next launch may then start
+    // scheduling its CTAs while this one runs.
+    grid_dependency_wait();
+    grid_launch_dependents();
+
     const int unit = blockIdx.x / splits;
     const int split = blockIdx.x - unit * splits;
     const int g = threadIdx.x / LPR;
@@ -58,68 +154,60 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
     const uint4 *knu = k_new + (size_t)unit * LPR;
     const uint4 *vnu = v_new + (size_t)unit * LPR;
 
-    float qf[8];
-    unpack8(q[(size_t)unit * LPR + l], qf);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) qf[i] *= scale_log2e;
-
-    const int rows = len + 1;
-    const int per = (rows + splits - 1) / splits;
-    const int r0 = split * per, r1 = min(r0 + per, rows);
-
-    float m = -INFINITY, lsum = 0.f, acc[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-
-    for (int j0 = r0 + g * kRowsPerIter; j0 < r1; j0 += G * kRowsPerIter) {
-        uint4 rk[kRowsPerIter], rv[kRowsPerIter];
-#pragma unroll
-        for (int r = 0; r < kRowsPerIter; ++r) {
-            const int j = j0 + r;
-            if (j < r1) {
-                const uint4 *pk = (j < len) ? Kcu + (size_t)j * LPR : knu;
-                const uint4 *pv = (j < len) ? Vcu + (size_t)j * LPR : vnu;
-                rk[r] = ld_row(pk + l);
-                rv[r] = ld_row(pv + l);
-            } else {
-                rk[r] = make_uint4(0, 0, 0, 0);
-                rv[r] = make_uint4(0, 0, 0, 0);
-            }
-        }
-        float s[kRowsPerIter];
-#pragma unroll
-        for (int r = 0; r < kRowsPerIter; ++r) {
-            float f[8];
-            unpack8(rk[r], f);
-            float d = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) d = fmaf(qf[i], f[i], d);
-#pragma unroll
-            for (int o = LPR / 2; o >= 1; o >>= 1) d += __shfl_xor_sync(gmask, d, o);
-            s[r] = (j0 + r < r1) ? d : -INFINITY;
-        }
-        float mn = m;
-#pragma unroll
-        for (int r = 0; r < kRowsPerIter; ++r) mn = fmaxf(mn, s[r]);
-        const float corr = fast_exp2(m - mn);      // first pass: exp2(-inf) = 0
-        m = mn;
-        lsum *= corr;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] *= corr;
-#pragma unroll
-        for (int r = 0; r < kRowsPerIter; ++r) {
-            const float p = fast_exp2(s[r] - mn);
-            lsum += p;
-            float f[8];
-            unpack8(rv[r], f);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = fmaf(p, f[i], acc[i]);
-        }
+    float2 q2[4];
+    {
+        const uint4 qv = q[(size_t)unit * LPR + l];
+        const float2 s2 = make_float2(scale_log2e, scale_log2e), z2 = make_float2(0.f, 0.f);
+        q2[0] = __ffma2_rn(unpack2(qv.x), s2, z2);
+        q2[1] = __ffma2_rn(unpack2(qv.y), s2, z2);
+        q2[2] = __ffma2_rn(unpack2(qv.z), s2, z2);
+        q2[3] = __ffma2_rn(unpack2(qv.w), s2, z2);
     }
 
-    if (l == 0) { sm_m[g] = m; sm_l[g] = lsum; }
+    // cached rows of this split: [r0, r1); the last split also takes the new row
+    const int per = (len + splits - 1) / splits;
+    const int r0 = min(split * per, len), r1 = min(r0 + per, len);
+    const int nfull = (r1 - r0) / kBlk;
+
+    GroupState st;
+    st.m = -INFINITY;
+    st.lsum = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) sm_acc[g][l * 8 + i] = acc[i];
+    for (int i = 0; i < 4; ++i) st.acc[i] = make_float2(0.f, 0.f);
+
+    const uint4 *Kl = Kcu + l, *Vl = Vcu + l;
+    for (int b = g; b < nfull; b += G) process_block<LPR, false>(st, q2, Kl, Vl, r0 + b * kBlk, r1, l, gmask);
+    if (r0 + nfull * kBlk < r1 && (nfull % G) == g)
+        process_block<LPR, true>(st, q2, Kl, Vl, r0 + nfull * kBlk, r1, l, gmask);
+
+    // per-lane partial sums -> group sum (rows are owned by LPR/8 lanes each)
+    float lsum = st.lsum;
+#pragma unroll
+    for (int o = LPR / 2; o >= 1; o >>= 1) lsum += __shfl_xor_sync(gmask, lsum, o);
+    lsum *= (float)kBlk / (float)LPR;
+
+    if (split == splits - 1 && g == G - 1) {
+        // the step's own (k_new, v_new) row, straight from the inputs
+        const uint4 kn = ld_row(knu + l), vn = ld_row(vnu + l);
+        float sc = dot8(q2, kn);
+#pragma unroll
+        for (int o = LPR / 2; o >= 1; o >>= 1) sc += __shfl_xor_sync(gmask, sc, o);
+        const float mn = fmaxf(st.m, sc);
+        const float corr = fast_exp2(st.m - mn), p = fast_exp2(sc - mn);
+        st.m = mn;
+        lsum = fmaf(lsum, corr, p);
+        const float2 c2 = make_float2(corr, corr), z2 = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) st.acc[i] = __ffma2_rn(st.acc[i], c2, z2);
+        axpy8(st.acc, p, vn);
+    }
+
+    if (l == 0) { sm_m[g] = st.m; sm_l[g] = lsum; }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        sm_acc[g][l * 8 + 2 * i] = st.acc[i].x;
+        sm_acc[g][l * 8 + 2 * i + 1] = st.acc[i].y;
+    }
     __syncthreads();   // also orders every cache read of this CTA before the slot write below
 
     for (int d = threadIdx.x; d < D; d += kDecThreads) {
@@ -156,6 +244,8 @@ __global__ void combine_kernel(const float *__restrict__ partials, int splits,
                                uint4 *Kc, uint4 *Vc, int cap, int write_slot, __nv_bfloat16 *__restrict__ out)
 {
     constexpr int D = LPR * 8;
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int unit = blockIdx.x;
     const int d = threadIdx.x;
     const float *p = partials + (size_t)unit * splits * (D + 2);
@@ -193,31 +283,47 @@ int decode_splits(int units, int rows)
     return s;
 }
 
+// Kernel launch that allows the launch latency of consecutive decode steps to overlap
+// (the kernels themselves wait for their predecessor before touching memory).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+template <int LPR>
+cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc, int units,
+                            int cap, int len, int write_slot, float sl2, void *out, float *partials, int splits,
+                            cudaStream_t stream)
+{
+    cudaError_t e = launch_overlapped(decode_kernel<LPR>, (unsigned)(units * splits), (unsigned)kDecThreads, stream,
+                                      (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc,
+                                      (uint4 *)Vc, cap, len, write_slot, sl2, (__nv_bfloat16 *)out, partials, splits);
+    if (e != cudaSuccess || splits == 1) return e;
+    return launch_overlapped(combine_kernel<LPR>, (unsigned)units, (unsigned)(LPR * 8), stream,
+                             (const float *)partials, splits, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc,
+                             (uint4 *)Vc, cap, write_slot, (__nv_bfloat16 *)out);
+}
+
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
                           int units, int D, int cap, int len, int write_slot, float scale, void *out,
                           float *partials, int splits, cudaStream_t stream)
 {
     const float sl2 = scale * 1.4426950408889634f;
-    const long long grid = (long long)units * splits;
-    if (grid > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    if (D == 128) {
-        decode_kernel<16><<<(unsigned)grid, kDecThreads, 0, stream>>>(
-            (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap, len,
-            write_slot, sl2, (__nv_bfloat16 *)out, partials, splits);
-        if (splits > 1)
-            combine_kernel<16><<<units, 128, 0, stream>>>(partials, splits, (const uint4 *)k_new,
-                                                          (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap,
-                                                          write_slot, (__nv_bfloat16 *)out);
-    } else {
-        decode_kernel<8><<<(unsigned)grid, kDecThreads, 0, stream>>>(
-            (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap, len,
-            write_slot, sl2, (__nv_bfloat16 *)out, partials, splits);
-        if (splits > 1)
-            combine_kernel<8><<<units, 64, 0, stream>>>(partials, splits, (const uint4 *)k_new,
-                                                         (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap,
-                                                         write_slot, (__nv_bfloat16 *)out);
-    }
-    return cudaGetLastError();
+    if ((long long)units * splits > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    if (D == 128)
+        return launch_decode_t<16>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, sl2, out, partials, splits, stream);
+    return launch_decode_t<8>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, sl2, out, partials, splits, stream);
 }
 
 }  // namespace ec
