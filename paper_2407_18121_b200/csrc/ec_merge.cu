@@ -20,11 +20,13 @@ namespace {
 #define EC_MERGE_ROWS_PER_CTA 256
 #endif
 #ifndef EC_MERGE_UNROLL
-#define EC_MERGE_UNROLL 4
+#define EC_MERGE_UNROLL 8
 #endif
 constexpr int kMergeThreads = EC_MERGE_THREADS;
 constexpr int kRowsPerCta = EC_MERGE_ROWS_PER_CTA;
 constexpr int kUnroll = EC_MERGE_UNROLL;
+
+__device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16lo(w), bf16hi(w)); }
 
 // First row of bucket k (Eq. 2): one past the midpoint between anchors k-1 and k.
 __device__ __forceinline__ int bucket_lo(const int32_t *anch, int k)
@@ -57,6 +59,9 @@ merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int
     const int g = threadIdx.x / LPR;
     const int l = threadIdx.x - g * LPR;
 
+    // launched with programmatic stream serialization right behind the selection kernel:
+    // wait for its anchors before the first global access
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int32_t *ap = anchor_pos + (size_t)unit * C;
     for (int k = threadIdx.x; k < C; k += kMergeThreads) anch[k] = ap[k];
     __syncthreads();
@@ -76,35 +81,48 @@ merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int
     int lo = bucket_lo(anch, k);
     const int last = (k_end == C) ? T - 1 : bucket_lo(anch, k_end) - 1;   // last row this group reads
     int hi = (k == C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
-    float ak[8], av[8];
+    const float2 one2 = make_float2(1.f, 1.f), zero2 = make_float2(0.f, 0.f);
+    float2 ak[4], av[4];                             // packed fp32 pairs: element 2i, 2i+1 of this lane's 8
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { ak[i] = 0.f; av[i] = 0.f; }
+    for (int i = 0; i < 4; ++i) { ak[i] = zero2; av[i] = zero2; }
 
     for (int t = lo; t <= last; t += kUnroll) {
         uint4 rk[kUnroll], rv[kUnroll];
 #pragma unroll
         for (int j = 0; j < kUnroll; ++j) {
-            if (t + j <= last) {
-                rk[j] = ldg_stream(Ku + (size_t)(t + j) * LPR);
-                rv[j] = ldg_stream(Vu + (size_t)(t + j) * LPR);
-            }
+            const int tj = min(t + j, last);         // rows past the group's range: reload the last row, unused
+            rk[j] = ldg_stream(Ku + (size_t)tj * LPR);
+            rv[j] = ldg_stream(Vu + (size_t)tj * LPR);
         }
 #pragma unroll
         for (int j = 0; j < kUnroll; ++j) {
             if (t + j <= last) {
-                float fk[8], fv[8];
-                unpack8(rk[j], fk);
-                unpack8(rv[j], fv);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { ak[i] += fk[i]; av[i] += fv[i]; }
+                ak[0] = __ffma2_rn(unpack2(rk[j].x), one2, ak[0]);
+                ak[1] = __ffma2_rn(unpack2(rk[j].y), one2, ak[1]);
+                ak[2] = __ffma2_rn(unpack2(rk[j].z), one2, ak[2]);
+                ak[3] = __ffma2_rn(unpack2(rk[j].w), one2, ak[3]);
+                av[0] = __ffma2_rn(unpack2(rv[j].x), one2, av[0]);
+                av[1] = __ffma2_rn(unpack2(rv[j].y), one2, av[1]);
+                av[2] = __ffma2_rn(unpack2(rv[j].z), one2, av[2]);
+                av[3] = __ffma2_rn(unpack2(rv[j].w), one2, av[3]);
                 if (t + j == hi) {
-                    const float inv = 1.0f / (float)(hi - lo + 1);      // exactly 1 for a singleton bucket
+                    const int cnt = hi - lo + 1;
+                    const float inv = (cnt == 1) ? 1.0f : __frcp_rn((float)cnt);   // a singleton stays bit-exact
+                    const float2 inv2 = make_float2(inv, inv);
+                    uint4 ok, ov;
+                    float2 m;
+                    m = __ffma2_rn(ak[0], inv2, zero2); ok.x = pack2(m.x, m.y);
+                    m = __ffma2_rn(ak[1], inv2, zero2); ok.y = pack2(m.x, m.y);
+                    m = __ffma2_rn(ak[2], inv2, zero2); ok.z = pack2(m.x, m.y);
+                    m = __ffma2_rn(ak[3], inv2, zero2); ok.w = pack2(m.x, m.y);
+                    m = __ffma2_rn(av[0], inv2, zero2); ov.x = pack2(m.x, m.y);
+                    m = __ffma2_rn(av[1], inv2, zero2); ov.y = pack2(m.x, m.y);
+                    m = __ffma2_rn(av[2], inv2, zero2); ov.z = pack2(m.x, m.y);
+                    m = __ffma2_rn(av[3], inv2, zero2); ov.w = pack2(m.x, m.y);
+                    Kcu[(size_t)k * LPR] = ok;
+                    Vcu[(size_t)k * LPR] = ov;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) { ak[i] *= inv; av[i] *= inv; }
-                    Kcu[(size_t)k * LPR] = pack8(ak);
-                    Vcu[(size_t)k * LPR] = pack8(av);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) { ak[i] = 0.f; av[i] = 0.f; }
+                    for (int i = 0; i < 4; ++i) { ak[i] = zero2; av[i] = zero2; }
                     ++k;
                     lo = hi + 1;
                     hi = (k >= C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
@@ -112,6 +130,29 @@ merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int
             }
         }
     }
+}
+
+template <int LPR>
+cudaError_t launch_merge_t(const void *K, const void *V, const int32_t *anchor_pos, unsigned grid, int T, int n_keep,
+                           int slices, void *Kc, void *Vc, int cap, cudaStream_t stream)
+{
+    const size_t smem = (size_t)n_keep * sizeof(int32_t);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(merge_kernel<LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kMergeThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, merge_kernel<LPR>, (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, slices,
+                              (uint4 *)Kc, (uint4 *)Vc, cap);
 }
 
 }  // namespace
@@ -122,23 +163,8 @@ cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos
     const int slices = (T + kRowsPerCta - 1) / kRowsPerCta;
     const long long grid = (long long)units * slices;
     if (grid > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    const size_t smem = (size_t)n_keep * sizeof(int32_t);
-    if (D == 128) {
-        if (smem > 48 * 1024) {
-            cudaError_t e = cudaFuncSetAttribute(merge_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return e;
-        }
-        merge_kernel<16><<<(unsigned)grid, kMergeThreads, smem, stream>>>(
-            (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, slices, (uint4 *)Kc, (uint4 *)Vc, cap);
-    } else {
-        if (smem > 48 * 1024) {
-            cudaError_t e = cudaFuncSetAttribute(merge_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return e;
-        }
-        merge_kernel<8><<<(unsigned)grid, kMergeThreads, smem, stream>>>(
-            (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, slices, (uint4 *)Kc, (uint4 *)Vc, cap);
-    }
-    return cudaGetLastError();
+    if (D == 128) return launch_merge_t<16>(K, V, anchor_pos, (unsigned)grid, T, n_keep, slices, Kc, Vc, cap, stream);
+    return launch_merge_t<8>(K, V, anchor_pos, (unsigned)grid, T, n_keep, slices, Kc, Vc, cap, stream);
 }
 
 }  // namespace ec

@@ -126,6 +126,8 @@ select_kernel(const float *__restrict__ scores, int T, int C, int protect_ends, 
     }
     __syncthreads();
 
+    // the merge kernel behind this one may start scheduling; it waits for this grid to finish
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int r = 0; r < replicate; ++r) {
         int32_t *ap = anchor_pos + (unit * replicate + r) * C;
         for (int k = tid; k < C; k += kSelThreads) ap[k] = anch[k];
