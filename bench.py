@@ -313,7 +313,9 @@ def run_ours(args, w: wl.Workload):
     mrg_gbs = mrg_bytes / (mrg_ms * 1e-3) / 1e9
     imp_flops = 2.0 * D * T * (T + 1) * units   # two passes, each 2*D flops for T(T+1)/2 causal scores
     imp_tflops = imp_flops / (imp_ms * 1e-3) / 1e12
-    splits = 1 if units >= 592 else None
+    # kernels per pass: two importance passes, selection, merge, and one decode kernel per token
+    # (plus one combine kernel per token when a unit's rows are split over several CTAs)
+    splits = max(1, min(-(-148 * 4 // units), -(-(C + 1) // 64)))
     launches_per_pass = 2 + 2 + S * (1 if splits == 1 else 2)
 
     line = {
