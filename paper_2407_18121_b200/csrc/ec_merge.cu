@@ -45,19 +45,24 @@ __device__ __forceinline__ int first_bucket_from(const int32_t *anch, int C, int
     return lo;
 }
 
-// LPR = lanes per row = D / 8 (each lane holds 8 bf16 = 16 bytes of a row).
+// LPR = lanes per row = D / 8 (each lane holds 8 bf16 = 16 bytes of a row). A lane group is
+// 2*LPR lanes: the first LPR stream the K row of a position, the other LPR its V row, so both
+// halves see the same bucket boundaries (for D = 128 a group is exactly one warp: no divergence).
 // grid.x = units * slices. Dynamic shared memory: the unit's C anchors.
 template <int LPR>
 __global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int32_t *__restrict__ anchor_pos,
              int T, int C, int slices, uint4 *__restrict__ Kc, uint4 *__restrict__ Vc, int cap)
 {
-    constexpr int G = kMergeThreads / LPR;          // lane groups per CTA
+    constexpr int GL = 2 * LPR;                     // lanes per group
+    constexpr int G = kMergeThreads / GL;           // lane groups per CTA
     extern __shared__ int32_t anch[];
     const int unit = blockIdx.x / slices;
     const int slice = blockIdx.x - unit * slices;
-    const int g = threadIdx.x / LPR;
-    const int l = threadIdx.x - g * LPR;
+    const int g = threadIdx.x / GL;
+    const int gl = threadIdx.x - g * GL;
+    const bool is_v = gl >= LPR;
+    const int l = is_v ? gl - LPR : gl;
 
     // launched with programmatic stream serialization right behind the selection kernel:
     // wait for its anchors before the first global access
@@ -73,56 +78,42 @@ merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int
     const int k_end = first_bucket_from(anch, C, rb);
     if (k >= k_end) return;
 
-    const uint4 *Ku = K + (size_t)unit * T * LPR + l;
-    const uint4 *Vu = V + (size_t)unit * T * LPR + l;
-    uint4 *Kcu = Kc + (size_t)unit * cap * LPR + l;
-    uint4 *Vcu = Vc + (size_t)unit * cap * LPR + l;
+    const uint4 *src = (is_v ? V : K) + (size_t)unit * T * LPR + l;
+    uint4 *dst = (is_v ? Vc : Kc) + (size_t)unit * cap * LPR + l;
 
     int lo = bucket_lo(anch, k);
     const int last = (k_end == C) ? T - 1 : bucket_lo(anch, k_end) - 1;   // last row this group reads
     int hi = (k == C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
     const float2 one2 = make_float2(1.f, 1.f), zero2 = make_float2(0.f, 0.f);
-    float2 ak[4], av[4];                             // packed fp32 pairs: element 2i, 2i+1 of this lane's 8
+    float2 acc[4];                                   // packed fp32 pairs: elements 2i, 2i+1 of this lane's 8
 #pragma unroll
-    for (int i = 0; i < 4; ++i) { ak[i] = zero2; av[i] = zero2; }
+    for (int i = 0; i < 4; ++i) acc[i] = zero2;
 
     for (int t = lo; t <= last; t += kUnroll) {
-        uint4 rk[kUnroll], rv[kUnroll];
+        uint4 rw[kUnroll];
 #pragma unroll
-        for (int j = 0; j < kUnroll; ++j) {
-            const int tj = min(t + j, last);         // rows past the group's range: reload the last row, unused
-            rk[j] = ldg_stream(Ku + (size_t)tj * LPR);
-            rv[j] = ldg_stream(Vu + (size_t)tj * LPR);
-        }
+        for (int j = 0; j < kUnroll; ++j)            // rows past the range: reload the last row, unused
+            rw[j] = ldg_stream(src + (size_t)min(t + j, last) * LPR);
 #pragma unroll
         for (int j = 0; j < kUnroll; ++j) {
             if (t + j <= last) {
-                ak[0] = __ffma2_rn(unpack2(rk[j].x), one2, ak[0]);
-                ak[1] = __ffma2_rn(unpack2(rk[j].y), one2, ak[1]);
-                ak[2] = __ffma2_rn(unpack2(rk[j].z), one2, ak[2]);
-                ak[3] = __ffma2_rn(unpack2(rk[j].w), one2, ak[3]);
-                av[0] = __ffma2_rn(unpack2(rv[j].x), one2, av[0]);
-                av[1] = __ffma2_rn(unpack2(rv[j].y), one2, av[1]);
-                av[2] = __ffma2_rn(unpack2(rv[j].z), one2, av[2]);
-                av[3] = __ffma2_rn(unpack2(rv[j].w), one2, av[3]);
+                acc[0] = __ffma2_rn(unpack2(rw[j].x), one2, acc[0]);
+                acc[1] = __ffma2_rn(unpack2(rw[j].y), one2, acc[1]);
+                acc[2] = __ffma2_rn(unpack2(rw[j].z), one2, acc[2]);
+                acc[3] = __ffma2_rn(unpack2(rw[j].w), one2, acc[3]);
                 if (t + j == hi) {
                     const int cnt = hi - lo + 1;
                     const float inv = (cnt == 1) ? 1.0f : __frcp_rn((float)cnt);   // a singleton stays bit-exact
                     const float2 inv2 = make_float2(inv, inv);
-                    uint4 ok, ov;
+                    uint4 o;
                     float2 m;
-                    m = __ffma2_rn(ak[0], inv2, zero2); ok.x = pack2(m.x, m.y);
-                    m = __ffma2_rn(ak[1], inv2, zero2); ok.y = pack2(m.x, m.y);
-                    m = __ffma2_rn(ak[2], inv2, zero2); ok.z = pack2(m.x, m.y);
-                    m = __ffma2_rn(ak[3], inv2, zero2); ok.w = pack2(m.x, m.y);
-                    m = __ffma2_rn(av[0], inv2, zero2); ov.x = pack2(m.x, m.y);
-                    m = __ffma2_rn(av[1], inv2, zero2); ov.y = pack2(m.x, m.y);
-                    m = __ffma2_rn(av[2], inv2, zero2); ov.z = pack2(m.x, m.y);
-                    m = __ffma2_rn(av[3], inv2, zero2); ov.w = pack2(m.x, m.y);
-                    Kcu[(size_t)k * LPR] = ok;
-                    Vcu[(size_t)k * LPR] = ov;
+                    m = __ffma2_rn(acc[0], inv2, zero2); o.x = pack2(m.x, m.y);
+                    m = __ffma2_rn(acc[1], inv2, zero2); o.y = pack2(m.x, m.y);
+                    m = __ffma2_rn(acc[2], inv2, zero2); o.z = pack2(m.x, m.y);
+                    m = __ffma2_rn(acc[3], inv2, zero2); o.w = pack2(m.x, m.y);
+                    dst[(size_t)k * LPR] = o;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) { ak[i] = zero2; av[i] = zero2; }
+                    for (int i = 0; i < 4; ++i) acc[i] = zero2;
                     ++k;
                     lo = hi + 1;
                     hi = (k >= C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
