@@ -35,6 +35,24 @@ METRIC = "decode tokens/s on merged KV (whole pass: importance + select/merge + 
 UNIT = "tokens/s"
 
 
+# DRAM bytes (read + write) of one decode_kernel launch from the ncu capture summarised in
+# profiles/decode_kernel_llava7b_b1_ncu.md, keyed by workload; valid only for the kernel source it was
+# taken on (sha1 prefix of csrc/ec_decode.cu), otherwise reported as null.
+DECODE_TRAFFIC = {"source_sha1": "97a0d9b0252a", "llava7b_b1": 173.9e6}
+
+
+def decode_traffic(workload: str):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2407_18121_b200", "csrc", "ec_decode.cu")
+    try:
+        digest = hashlib.sha1(open(path, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if not digest.startswith(DECODE_TRAFFIC["source_sha1"]):
+        return None
+    return DECODE_TRAFFIC.get(workload)
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -61,7 +79,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -184,6 +202,30 @@ def workload_config(w: wl.Workload):
             "l2": "inputs larger than L2 (prompt Q/K/V and the compacted cache each exceed 126 MB per pass)"}
 
 
+# ----------------------------------------------------------------------------- rank logic
+
+def rank_workload(w: wl.Workload, rank: int) -> wl.Workload:
+    """The batch a rank works on: same shapes, its own seed. Ranks never exchange data."""
+    import dataclasses
+    return dataclasses.replace(w, seed=w.seed + 1000 * rank)
+
+
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(x) for x in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_tokens_per_s(w: wl.Workload, world: int, ms_per_pass: float) -> float:
+    """Every rank generates batch * decode_steps tokens per pass; the job's time is the slowest rank's."""
+    return w.batch * w.decode_steps * world / (ms_per_pass * 1e-3)
+
+
 # ----------------------------------------------------------------------------- GPU leg
 
 def run_ours(args, w: wl.Workload):
@@ -210,8 +252,7 @@ def run_ours(args, w: wl.Workload):
     ec.lib()
 
     # every rank holds its own batch of independent problems (weak scaling, no exchange)
-    import dataclasses
-    wr = dataclasses.replace(w, seed=w.seed + 1000 * rank)
+    wr = rank_workload(w, rank)
     N, H, T, D, S = wr.N, wr.heads, wr.prompt_len, wr.head_dim, wr.decode_steps
     Qb, Kb, Vb = wl.prompt(wr)
     qb, kb, vb = wl.decode_inputs(wr)
@@ -292,10 +333,7 @@ def run_ours(args, w: wl.Workload):
     d2h = d2h_b + anchors_h.numel() * 4
 
     ms_per_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms = t.tolist()
+    ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms = max_over_ranks([ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms], "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -303,7 +341,7 @@ def run_ours(args, w: wl.Workload):
 
     peaks = measured_peaks()
     tokens = w.batch * S * world
-    value = tokens / (ms_per_step * 1e-3)
+    value = whole_job_tokens_per_s(w, world, ms_per_step)
     # algorithmic bytes of one decode launch: every cached K and V row once, q/k_new/v_new in,
     # out and the overwritten slot (K and V row) out
     dec_bytes = units * (2 * C * D * 2 + 3 * D * 2 + D * 2 + 2 * D * 2)
@@ -328,7 +366,8 @@ def run_ours(args, w: wl.Workload):
         "decode_only_tokens_per_s": w.batch * S * world / (dec_ms * 1e-3),
         "roofline": {"kernel": "decode_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "frac_of_nominal_8TBs": dec_gbs / 8000.0, "bytes_per_launch": dec_bytes, "traffic": None},
+                     "frac_of_nominal_8TBs": dec_gbs / 8000.0, "bytes_per_launch": dec_bytes,
+                     "traffic": decode_traffic(w.name)},
         "merge": {"achieved": mrg_gbs, "unit": "GB/s", "frac": mrg_gbs / peaks["hbm_gbs"],
                   "frac_of_nominal_8TBs": mrg_gbs / 8000.0, "bytes_per_call": mrg_bytes,
                   "note": "whole ec_select_merge call (selection + merge kernels)"},
@@ -352,7 +391,7 @@ def run_ours(args, w: wl.Workload):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llava7b_b1", choices=list(wl.WORKLOADS))

@@ -44,6 +44,8 @@ class ElasticCacheSession:
         self.ws_dec = torch.empty(ec.ec_decode_workspace(self.cache), dtype=torch.uint8, device=dev)
         self._stage = None      # device staging for the *_host calls, allocated on first use
         self._dstage = None
+        self._up = None         # side streams of decode_host
+        self._down = None
 
     # ---- device-resident inputs ------------------------------------------------------
     def compress(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor) -> None:
@@ -85,14 +87,37 @@ class ElasticCacheSession:
         return 3 * Q_host.numel() * Q_host.element_size()
 
     def decode_host(self, q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor,
-                    out_host: torch.Tensor):
-        """decode() from pinned host tensors [steps, N, H, D]; writes out_host. Returns (h2d, d2h) bytes."""
+                    out_host: torch.Tensor, chunk: int = 64):
+        """decode() from pinned host tensors [steps, N, H, D]; writes out_host. Returns (h2d, d2h) bytes.
+
+        The steps are processed in chunks: the upload of the next chunk's inputs and the download of
+        the previous chunk's outputs run on two side streams while the current chunk decodes."""
         steps = q_host.shape[0]
         q, k, v, out = (t[:steps] for t in self._decode_staging(steps))
-        q.copy_(q_host, non_blocking=True)
-        k.copy_(k_host, non_blocking=True)
-        v.copy_(v_host, non_blocking=True)
-        self.decode(q, k, v, out)
-        out_host.copy_(out, non_blocking=True)
+        cur = torch.cuda.current_stream()
+        if self._up is None:
+            self._up, self._down = torch.cuda.Stream(), torch.cuda.Stream()
+        up, down = self._up, self._down
+        up.wait_stream(cur)                     # staging buffers may still be read by earlier work
+        down.wait_stream(cur)
+        bounds = [(a, min(a + chunk, steps)) for a in range(0, steps, chunk)]
+        ready = []
+        with torch.cuda.stream(up):
+            for a, b in bounds:
+                q[a:b].copy_(q_host[a:b], non_blocking=True)
+                k[a:b].copy_(k_host[a:b], non_blocking=True)
+                v[a:b].copy_(v_host[a:b], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(up)
+                ready.append(ev)
+        for (a, b), ev in zip(bounds, ready):
+            cur.wait_event(ev)
+            self.decode(q[a:b], k[a:b], v[a:b], out[a:b])
+            done = torch.cuda.Event()
+            done.record(cur)
+            with torch.cuda.stream(down):
+                down.wait_event(done)
+                out_host[a:b].copy_(out[a:b], non_blocking=True)
+        cur.wait_stream(down)
         nb = q_host.numel() * q_host.element_size()
         return 3 * nb, nb
