@@ -86,6 +86,18 @@ int ec_importance(const void *Q_dev, const void *K_dev, float *scores_dev, float
                   void *ws_dev, size_t ws_bytes, void *stream);
 
 /*
+ * The same importance when the caller already holds every query row's log-sum-exp, as a
+ * prefill attention kernel produces it (the paper takes the attention probabilities from
+ * the model's own forward pass, Algorithm 1 "Input"): only the column-sum pass runs, which
+ * halves the contraction work.
+ *   lse_dev   fp32 [N, H, T], natural log of sum_{n<=m} exp(scale*<q_m,k_n>), same `scale`  (in)
+ * Other arguments, workspace size and limits as ec_importance; additionally N*H <= 65535.
+ */
+int ec_importance_from_lse(const void *Q_dev, const void *K_dev, const float *lse_dev, float *scores_dev,
+                           int N, int H, int T, int D, float scale,
+                           void *ws_dev, size_t ws_bytes, void *stream);
+
+/*
  * Synchronises `stream` and reports what the kernels recorded in the workspace's status
  * word: EC_OK, or EC_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are
  * then undefined but no out-of-bounds access happened). EC_ERR_CUDA on a runtime error.
@@ -126,6 +138,28 @@ int ec_select_merge(const void *K_dev, const void *V_dev, const float *scores_de
                     int32_t *anchor_pos_dev, int32_t *bucket_len_dev,
                     void *ws_dev, size_t ws_bytes, void *stream);
 
+/*
+ * The general form of ec_select_merge, covering the variants of the paper's ablations
+ * (Sec. 4.3: importance population; cache eviction versus cache merging):
+ *   share       how many consecutive units rank one common score vector (the mean of their
+ *               scores): 1 = head-wise, H = layer-wise, layers*H = one selection per sequence
+ *               ("identical" for all layers; problems n = b*layers + l must be layer-minor).
+ *               N*H must be a multiple of share; N*H/share <= 65535 when share > 1.
+ *   compaction  EC_COMPACT_MERGE: bucket means (Eq. 3).  EC_COMPACT_EVICT: the kept rows are
+ *               the anchors' own rows and all other rows are dropped.
+ * Everything else as ec_select_merge, which is this call with share = 1 or H and
+ * EC_COMPACT_MERGE. Workspace: ec_select_compact_workspace.
+ */
+typedef enum { EC_COMPACT_MERGE = 0, EC_COMPACT_EVICT = 1 } ec_compaction;
+
+size_t ec_select_compact_workspace(int N, int H, int T, int D, int n_keep, int share);
+
+int ec_select_compact(const void *K_dev, const void *V_dev, const float *scores_dev,
+                      int N, int H, int T, int D, int n_keep, int share, int protect_ends, int compaction,
+                      void *Kc_dev, void *Vc_dev, int cap,
+                      int32_t *anchor_pos_dev, int32_t *bucket_len_dev,
+                      void *ws_dev, size_t ws_bytes, void *stream);
+
 /* ---------------------------------------------------------------- decode ------------ */
 
 /*
@@ -143,11 +177,38 @@ typedef struct {
     int offset;         /* rows that stay behind the truncation location (>= 1)          */
     int ring_head;      /* next ring slot to be reused, 0..offset-1                      */
     int64_t step;       /* decode steps taken                                            */
+    /* retention-ratio policy only (see ec_cache_init_ratio); zero / NULL otherwise      */
+    int policy;         /* EC_POLICY_FIXED or EC_POLICY_RATIO                            */
+    int recent_head;    /* position of the oldest entry in recent_slots_host             */
+    double keep_ratio;  /* retained fraction of all tokens seen                          */
+    int64_t n_tot;      /* tokens seen so far, prompt included                           */
+    int *recent_slots_host; /* caller-owned host array of `offset` ints: physical slots
+                               of the `offset` newest rows, kept as a ring               */
 } ec_cache;
+
+typedef enum {
+    EC_POLICY_FIXED = 0, /* the cache stays at `budget` rows: one row leaves every step  */
+    EC_POLICY_RATIO = 1  /* the budget follows keep_ratio * tokens seen (Sec. 3.3: the
+                            ratio is compared with a threshold after every new token)    */
+} ec_policy;
 
 /* Fills *c after validating: 2 <= budget <= cap, 0 <= len <= budget, 1 <= offset <= budget-1. */
 int ec_cache_init(ec_cache *c, void *Kc_dev, void *Vc_dev, int N, int H, int D, int cap,
                   int len, int budget, int offset);
+
+/*
+ * Retention-ratio policy (Sec. 3.3 "Output Generation"; Algorithm 1: del_num =
+ * int(seq_len - n * retained_fraction), evaluated after the new row was appended). A step
+ * removes the row at the fixed truncation location only when del_num >= 1; otherwise the
+ * cache grows by one row (up to cap; a step that would exceed cap returns EC_ERR_ARG).
+ *   len                rows valid now (e.g. n_keep after ec_select_merge), len >= offset
+ *   n_tot              tokens seen so far (the prompt length after the prompt call)
+ *   recent_slots_host  host array of `offset` ints owned by the caller; it must stay valid
+ *                      as long as *c is used. Rows that are no longer among the `offset`
+ *                      newest never move again, so only these slots have to be tracked.
+ */
+int ec_cache_init_ratio(ec_cache *c, void *Kc_dev, void *Vc_dev, int N, int H, int D, int cap,
+                        int len, int offset, double keep_ratio, int64_t n_tot, int *recent_slots_host);
 
 size_t ec_decode_workspace(const ec_cache *c);
 

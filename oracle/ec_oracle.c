@@ -139,6 +139,29 @@ void eco_layer_mean(const double *scores, int N, int H, int T, double *out)
         }
 }
 
+/* Population shared by `share` consecutive units (Sec. 3.2 "population types"; ablation on the
+ * importance population): share = 1 is head-wise, share = H is layer-wise, share = L*H makes one
+ * score vector per sequence ("identical" for all layers). scores [G*share, T] -> out [G, T]. */
+void eco_group_mean(const double *scores, int G, int share, int T, double *out)
+{
+    for (int g = 0; g < G; ++g)
+        for (int t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int j = 0; j < share; ++j) acc += scores[((size_t)g * share + j) * T + t];
+            out[(size_t)g * T + t] = acc / (double)share;
+        }
+}
+
+/* Eviction instead of merging (the ablation's "cache eviction" row): the kept rows are the
+ * anchors' own rows, everything else is dropped. X: bf16 [U, T, D]; anchors [U, C]; out [U, C, D]. */
+void eco_gather(const uint16_t *X, int U, int T, int D, const int32_t *anchors, int C, double *out)
+{
+    for (int u = 0; u < U; ++u)
+        for (int k = 0; k < C; ++k)
+            for (int c = 0; c < D; ++c)
+                out[((size_t)u * C + k) * D + c] = bf16_to_double(X[((size_t)u * T + anchors[(size_t)u * C + k]) * D + c]);
+}
+
 typedef struct {
     double score;
     int32_t pos;

@@ -30,6 +30,10 @@ _lib.eco_importance.restype = None
 _lib.eco_importance.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_double, _f64p, _f64p]
 _lib.eco_layer_mean.restype = None
 _lib.eco_layer_mean.argtypes = [_f64p, C.c_int, C.c_int, C.c_int, _f64p]
+_lib.eco_group_mean.restype = None
+_lib.eco_group_mean.argtypes = [_f64p, C.c_int, C.c_int, C.c_int, _f64p]
+_lib.eco_gather.restype = None
+_lib.eco_gather.argtypes = [_u16p, C.c_int, C.c_int, C.c_int, _i32p, C.c_int, _f64p]
 _lib.eco_select.restype = None
 _lib.eco_select.argtypes = [_f64p, C.c_int, C.c_int, C.c_int, C.c_int, _i32p]
 _lib.eco_buckets.restype = None
@@ -83,6 +87,28 @@ def layer_mean(scores: np.ndarray) -> np.ndarray:
     N, H, T = s.shape
     out = np.empty((N, T), np.float64)
     _lib.eco_layer_mean(_p(s, _f64p), N, H, T, _p(out, _f64p))
+    return out
+
+
+def group_mean(scores: np.ndarray, share: int) -> np.ndarray:
+    """scores float64 [U, T] with U a multiple of share -> [U // share, T]."""
+    s = np.ascontiguousarray(scores, np.float64)
+    U, T = s.shape
+    assert U % share == 0
+    out = np.empty((U // share, T), np.float64)
+    _lib.eco_group_mean(_p(s, _f64p), U // share, int(share), T, _p(out, _f64p))
+    return out
+
+
+def gather(X: np.ndarray, anchors: np.ndarray) -> np.ndarray:
+    """X uint16 [..., T, D]; anchors int32 [..., C] -> float64 [..., C, D] (the anchors' own rows)."""
+    X = _bits(X)
+    a = np.ascontiguousarray(anchors, np.int32)
+    T, D = X.shape[-2:]
+    Ck = a.shape[-1]
+    U = int(np.prod(X.shape[:-2], dtype=np.int64))
+    out = np.empty(X.shape[:-2] + (Ck, D), np.float64)
+    _lib.eco_gather(_p(X, _u16p), U, T, D, _p(a, _i32p), Ck, _p(out, _f64p))
     return out
 
 

@@ -22,9 +22,9 @@ EC_LAYER_SHARED = 1
 
 EXPORTS = (
     "ec_status_string", "ec_keep_count",
-    "ec_importance_workspace", "ec_importance", "ec_device_status",
-    "ec_select_merge_workspace", "ec_select_merge",
-    "ec_cache_init", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
+    "ec_importance_workspace", "ec_importance", "ec_importance_from_lse", "ec_device_status",
+    "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
+    "ec_cache_init", "ec_cache_init_ratio", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc",
 )
 
@@ -40,7 +40,9 @@ class ec_cache(C.Structure):
     _fields_ = [("Kc", C.c_void_p), ("Vc", C.c_void_p),
                 ("N", C.c_int), ("H", C.c_int), ("D", C.c_int), ("cap", C.c_int),
                 ("len", C.c_int), ("budget", C.c_int), ("offset", C.c_int),
-                ("ring_head", C.c_int), ("step", C.c_int64)]
+                ("ring_head", C.c_int), ("step", C.c_int64),
+                ("policy", C.c_int), ("recent_head", C.c_int), ("keep_ratio", C.c_double),
+                ("n_tot", C.c_int64), ("recent_slots_host", C.POINTER(C.c_int))]
 
 
 _lib = None
@@ -64,14 +66,23 @@ def lib() -> C.CDLL:
     L.ec_importance_workspace.argtypes = [i, i, i, i]
     L.ec_importance.restype = i
     L.ec_importance.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
+    L.ec_importance_from_lse.restype = i
+    L.ec_importance_from_lse.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
     L.ec_device_status.restype = i
     L.ec_device_status.argtypes = [vp, vp]
     L.ec_select_merge_workspace.restype = sz
     L.ec_select_merge_workspace.argtypes = [i, i, i, i, i, i]
     L.ec_select_merge.restype = i
     L.ec_select_merge.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, vp, vp, i, vp, vp, vp, sz, vp]
+    L.ec_select_compact_workspace.restype = sz
+    L.ec_select_compact_workspace.argtypes = [i, i, i, i, i, i]
+    L.ec_select_compact.restype = i
+    L.ec_select_compact.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, vp, vp, i, vp, vp, vp, sz, vp]
     L.ec_cache_init.restype = i
     L.ec_cache_init.argtypes = [C.POINTER(ec_cache), vp, vp, i, i, i, i, i, i, i]
+    L.ec_cache_init_ratio.restype = i
+    L.ec_cache_init_ratio.argtypes = [C.POINTER(ec_cache), vp, vp, i, i, i, i, i, i, C.c_double, C.c_int64,
+                                      C.POINTER(C.c_int)]
     L.ec_decode_workspace.restype = sz
     L.ec_decode_workspace.argtypes = [C.POINTER(ec_cache)]
     L.ec_decode_step.restype = i
@@ -126,6 +137,15 @@ def ec_importance(Q: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, lse: O
     _check(st, "ec_importance")
 
 
+def ec_importance_from_lse(Q: torch.Tensor, K: torch.Tensor, lse: torch.Tensor, scores: torch.Tensor,
+                           scale: float, ws: torch.Tensor) -> None:
+    """Importance from a known per-row log-sum-exp (fp32 [N,H,T], natural log): column-sum pass only."""
+    N, H, T, D = Q.shape
+    st = lib().ec_importance_from_lse(_ptr(Q), _ptr(K), _ptr(lse), _ptr(scores), N, H, T, D, float(scale),
+                                      _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_importance_from_lse")
+
+
 def ec_device_status(ws: torch.Tensor) -> int:
     return int(lib().ec_device_status(_ptr(ws), _stream()))
 
@@ -147,12 +167,48 @@ def ec_select_merge(K: torch.Tensor, V: torch.Tensor, scores: torch.Tensor, n_ke
     _check(st, "ec_select_merge")
 
 
+EC_COMPACT_MERGE = 0
+EC_COMPACT_EVICT = 1
+
+
+def ec_select_compact_workspace(N: int, H: int, T: int, D: int, n_keep: int, share: int) -> int:
+    return int(lib().ec_select_compact_workspace(N, H, T, D, n_keep, share))
+
+
+def ec_select_compact(K: torch.Tensor, V: torch.Tensor, scores: torch.Tensor, n_keep: int, share: int,
+                      protect_ends: bool, compaction: int, Kc: torch.Tensor, Vc: torch.Tensor,
+                      anchor_pos: torch.Tensor, bucket_len: Optional[torch.Tensor], ws: torch.Tensor) -> None:
+    """ec_select_merge with an explicit sharing width (`share` consecutive units rank one averaged score
+    vector) and a choice between bucket means (EC_COMPACT_MERGE) and plain eviction (EC_COMPACT_EVICT)."""
+    N, H, T, D = K.shape
+    cap = Kc.shape[2]
+    st = lib().ec_select_compact(_ptr(K), _ptr(V), _ptr(scores), N, H, T, D, int(n_keep), int(share),
+                                 int(bool(protect_ends)), int(compaction), _ptr(Kc), _ptr(Vc), cap,
+                                 _ptr(anchor_pos), _ptr(bucket_len), _ptr(ws), ws.numel() * ws.element_size(),
+                                 _stream())
+    _check(st, "ec_select_compact")
+
+
 def ec_cache_init(Kc: torch.Tensor, Vc: torch.Tensor, length: int, budget: int, offset: int) -> ec_cache:
     """Describe a compacted cache held in Kc, Vc: bf16 [N,H,cap,D] with `length` valid rows."""
     N, H, cap, D = Kc.shape
     c = ec_cache()
     st = lib().ec_cache_init(C.byref(c), _ptr(Kc), _ptr(Vc), N, H, D, cap, int(length), int(budget), int(offset))
     _check(st, "ec_cache_init")
+    return c
+
+
+def ec_cache_init_ratio(Kc: torch.Tensor, Vc: torch.Tensor, length: int, offset: int, keep_ratio: float,
+                        n_tot: int) -> ec_cache:
+    """Cache under the retention-ratio policy: it grows while length < keep_ratio * tokens seen and
+    evicts at the fixed truncation location otherwise. The host ring of recent slots is owned by
+    the returned object."""
+    N, H, cap, D = Kc.shape
+    c = ec_cache()
+    c._recent = (C.c_int * int(offset))()          # kept alive with the struct
+    st = lib().ec_cache_init_ratio(C.byref(c), _ptr(Kc), _ptr(Vc), N, H, D, cap, int(length), int(offset),
+                                   float(keep_ratio), int(n_tot), c._recent)
+    _check(st, "ec_cache_init_ratio")
     return c
 
 

@@ -69,7 +69,22 @@ int ec_importance(const void *Q, const void *K, float *scores, float *lse, int N
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || (lse && !aligned(lse, 16))) return EC_ERR_ALIGN;
     if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EC_ERR_ALIGN;
-    cudaError_t e = ec::launch_importance(Q, K, scores, lse, N, H, T, D, scale, ws, (cudaStream_t)stream);
+    cudaError_t e = ec::launch_importance(Q, K, scores, lse, nullptr, N, H, T, D, scale, ws, (cudaStream_t)stream);
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+int ec_importance_from_lse(const void *Q, const void *K, const float *lse, float *scores, int N, int H, int T, int D,
+                           float scale, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!Q || !K || !scores || !lse) return EC_ERR_NULL;
+    int st = check_shape(N, H, T, D);
+    if (st != EC_OK) return st;
+    if ((long long)N * H > 65535) return EC_ERR_SHAPE;
+    if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || !aligned(lse, 4)) return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    cudaError_t e = ec::launch_importance(Q, K, scores, nullptr, lse, N, H, T, D, scale, ws, (cudaStream_t)stream);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 
@@ -83,36 +98,54 @@ int ec_device_status(void *ws, void *stream)
     return word == 0 ? EC_OK : EC_ERR_TIMEOUT;
 }
 
-size_t ec_select_merge_workspace(int N, int H, int T, int D, int n_keep, int population)
+size_t ec_select_compact_workspace(int N, int H, int T, int D, int n_keep, int share)
 {
     if (check_shape(N, H, T, D) != EC_OK || n_keep < 1 || n_keep > T) return 0;
-    // layer-shared mode keeps the head-averaged scores [N, T]; a minimum keeps the pointer non-null
-    size_t mean = (population == EC_LAYER_SHARED) ? round256((size_t)N * T * sizeof(float)) : 0;
+    if (share < 1 || ((long long)N * H) % share != 0) return 0;
+    // a shared population keeps the averaged scores [N*H/share, T]; a minimum keeps the pointer non-null
+    size_t mean = (share > 1) ? round256((size_t)N * H / share * T * sizeof(float)) : 0;
     return 256 + mean;
+}
+
+int ec_select_compact(const void *K, const void *V, const float *scores, int N, int H, int T, int D, int n_keep,
+                      int share, int protect_ends, int compaction, void *Kc, void *Vc, int cap, int32_t *anchor_pos,
+                      int32_t *bucket_len, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!K || !V || !scores || !Kc || !Vc || !anchor_pos) return EC_ERR_NULL;
+    int st = check_shape(N, H, T, D);
+    if (st != EC_OK) return st;
+    if (n_keep < 1 || n_keep > T || cap < n_keep) return EC_ERR_ARG;
+    if (share < 1 || ((long long)N * H) % share != 0) return EC_ERR_ARG;
+    if (share > 1 && (long long)N * H / share > 65535) return EC_ERR_SHAPE;
+    if (compaction != EC_COMPACT_MERGE && compaction != EC_COMPACT_EVICT) return EC_ERR_ARG;
+    if ((long long)N * H * cap >= (1LL << 31)) return EC_ERR_SHAPE;
+    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(scores, 4) ||
+        !aligned(anchor_pos, 4) || (bucket_len && !aligned(bucket_len, 4)))
+        return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < ec_select_compact_workspace(N, H, T, D, n_keep, share)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    float *mean_ws = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = ec::launch_select(scores, N * H, T, n_keep, share, protect_ends ? 1 : 0, anchor_pos, bucket_len,
+                                      mean_ws, s);
+    if (e != cudaSuccess) return EC_ERR_CUDA;
+    if (compaction == EC_COMPACT_MERGE) e = ec::launch_merge(K, V, anchor_pos, N * H, T, D, n_keep, Kc, Vc, cap, s);
+    else e = ec::launch_gather(K, V, anchor_pos, N * H, T, D, n_keep, Kc, Vc, cap, s);
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+size_t ec_select_merge_workspace(int N, int H, int T, int D, int n_keep, int population)
+{
+    return ec_select_compact_workspace(N, H, T, D, n_keep, population == EC_LAYER_SHARED ? H : 1);
 }
 
 int ec_select_merge(const void *K, const void *V, const float *scores, int N, int H, int T, int D, int n_keep,
                     int population, int protect_ends, void *Kc, void *Vc, int cap, int32_t *anchor_pos,
                     int32_t *bucket_len, void *ws, size_t ws_bytes, void *stream)
 {
-    if (!K || !V || !scores || !Kc || !Vc || !anchor_pos) return EC_ERR_NULL;
-    int st = check_shape(N, H, T, D);
-    if (st != EC_OK) return st;
-    if (n_keep < 1 || n_keep > T || cap < n_keep) return EC_ERR_ARG;
     if (population != EC_PER_HEAD && population != EC_LAYER_SHARED) return EC_ERR_ARG;
-    if ((long long)N * H * cap >= (1LL << 31)) return EC_ERR_SHAPE;
-    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(scores, 4) ||
-        !aligned(anchor_pos, 4) || (bucket_len && !aligned(bucket_len, 4)))
-        return EC_ERR_ALIGN;
-    if (!ws || ws_bytes < ec_select_merge_workspace(N, H, T, D, n_keep, population)) return EC_ERR_WORKSPACE;
-    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
-    float *mean_ws = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
-    cudaStream_t s = (cudaStream_t)stream;
-    cudaError_t e = ec::launch_select(scores, N, H, T, n_keep, population, protect_ends ? 1 : 0, anchor_pos,
-                                      bucket_len, mean_ws, s);
-    if (e != cudaSuccess) return EC_ERR_CUDA;
-    e = ec::launch_merge(K, V, anchor_pos, N * H, T, D, n_keep, Kc, Vc, cap, s);
-    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+    return ec_select_compact(K, V, scores, N, H, T, D, n_keep, population == EC_LAYER_SHARED ? H : 1, protect_ends,
+                             EC_COMPACT_MERGE, Kc, Vc, cap, anchor_pos, bucket_len, ws, ws_bytes, stream);
 }
 
 int ec_cache_init(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, int cap, int len, int budget, int offset)
@@ -128,6 +161,34 @@ int ec_cache_init(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, int cap,
     c->len = len; c->budget = budget; c->offset = offset;
     c->ring_head = 0;
     c->step = 0;
+    c->policy = EC_POLICY_FIXED;
+    c->recent_head = 0;
+    c->keep_ratio = 0.0;
+    c->n_tot = 0;
+    c->recent_slots_host = nullptr;
+    return EC_OK;
+}
+
+int ec_cache_init_ratio(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, int cap, int len, int offset,
+                        double keep_ratio, int64_t n_tot, int *recent_slots)
+{
+    if (!c || !Kc || !Vc || !recent_slots) return EC_ERR_NULL;
+    if (N < 1 || H < 1 || (D != 64 && D != 128) || cap < 1) return EC_ERR_SHAPE;
+    if ((long long)N * H * cap >= (1LL << 31) || (long long)N * H >= (1LL << 24)) return EC_ERR_SHAPE;
+    if (!aligned(Kc, 16) || !aligned(Vc, 16)) return EC_ERR_ALIGN;
+    if (offset < 1 || len < offset || len > cap) return EC_ERR_ARG;
+    if (!(keep_ratio > 0.0 && keep_ratio <= 1.0) || n_tot < len) return EC_ERR_ARG;
+    c->Kc = Kc; c->Vc = Vc;
+    c->N = N; c->H = H; c->D = D; c->cap = cap;
+    c->len = len; c->budget = len; c->offset = offset;
+    c->ring_head = 0;
+    c->step = 0;
+    c->policy = EC_POLICY_RATIO;
+    c->recent_head = 0;
+    c->keep_ratio = keep_ratio;
+    c->n_tot = n_tot;
+    c->recent_slots_host = recent_slots;
+    for (int i = 0; i < offset; ++i) recent_slots[i] = len - offset + i;   // oldest first
     return EC_OK;
 }
 
@@ -144,18 +205,37 @@ int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache
 {
     if (!q || !k_new || !v_new || !c || !out || !evicted_slot) return EC_ERR_NULL;
     if (!c->Kc || !c->Vc) return EC_ERR_NULL;
-    if (c->budget < 2 || c->budget > c->cap || c->len < 0 || c->len > c->budget || c->offset < 1 ||
-        c->offset > c->budget - 1 || c->ring_head < 0 || c->ring_head >= c->offset)
+    const bool ratio = (c->policy == EC_POLICY_RATIO);
+    if (ratio) {
+        if (!c->recent_slots_host || c->offset < 1 || c->len < c->offset || c->len > c->cap || c->recent_head < 0 ||
+            c->recent_head >= c->offset || !(c->keep_ratio > 0.0 && c->keep_ratio <= 1.0))
+            return EC_ERR_ARG;
+    } else if (c->budget < 2 || c->budget > c->cap || c->len < 0 || c->len > c->budget || c->offset < 1 ||
+               c->offset > c->budget - 1 || c->ring_head < 0 || c->ring_head >= c->offset) {
         return EC_ERR_ARG;
+    }
     if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
     if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16)) return EC_ERR_ALIGN;
     if (!ws || ws_bytes < ec_decode_workspace(c)) return EC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EC_ERR_ALIGN;
 
-    // Fixed-point elimination: at budget, queue position len - offset leaves. Rows before the
-    // ring never move, so that queue position is always the ring's oldest slot.
+    // Fixed-point elimination: queue position len - offset leaves, i.e. the oldest of the
+    // `offset` newest rows. Older rows never move, so only the newest rows' slots are tracked:
+    // a ring over [budget-offset, budget) for the fixed budget, an explicit ring of slots
+    // when the cache may still grow.
     int slot, evicted;
-    if (c->len < c->budget) {
+    if (ratio) {
+        // Algorithm 1: del_num = int(seq_len - n * retained_fraction), after the append
+        const double del = (double)(c->len + 1) - (double)(c->n_tot + 1) * c->keep_ratio;
+        if ((int)del >= 1) {
+            slot = c->recent_slots_host[c->recent_head];
+            evicted = slot;
+        } else {
+            if (c->len >= c->cap) return EC_ERR_ARG;     // no room left to grow
+            slot = c->len;
+            evicted = -1;
+        }
+    } else if (c->len < c->budget) {
         slot = c->len;
         evicted = -1;
     } else {
@@ -168,8 +248,17 @@ int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache
     cudaError_t e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, scale,
                                       out, partials, splits, (cudaStream_t)stream);
     if (e != cudaSuccess) return EC_ERR_CUDA;
-    if (evicted >= 0) c->ring_head = (c->ring_head + 1) % c->offset;
-    else c->len += 1;
+    if (ratio) {
+        // the new row is now the newest; the ring's oldest entry either left or stops being tracked
+        c->recent_slots_host[c->recent_head] = slot;
+        c->recent_head = (c->recent_head + 1) % c->offset;
+        if (evicted < 0) c->len += 1;
+        c->n_tot += 1;
+    } else if (evicted >= 0) {
+        c->ring_head = (c->ring_head + 1) % c->offset;
+    } else {
+        c->len += 1;
+    }
     c->step += 1;
     *evicted_slot = evicted;
     if (slot_written) *slot_written = slot;

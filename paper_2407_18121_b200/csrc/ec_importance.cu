@@ -375,9 +375,18 @@ bool make_map(CUtensorMap *map, const void *ptr, int units, int T, int D)
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A caller-provided natural-log normaliser [units, T] -> the padded log2-domain layout pass 2 reads.
+__global__ void lse_import_kernel(const float *__restrict__ lse_nat, float *__restrict__ lse2, int T, int Tpad)
+{
+    const int unit = blockIdx.y;
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= Tpad) return;
+    lse2[(size_t)unit * Tpad + m] = (m < T) ? lse_nat[(size_t)unit * T + m] * kLog2e : INFINITY;
+}
+
 template <int D, int STAGES>
-cudaError_t launch_both(const CUtensorMap &mq, const CUtensorMap &mk, int units, int T, int nt, float c, float *lse2,
-                        float *lse_out, float *scores, int *status, cudaStream_t stream)
+cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int units, int T, int nt, float c, float *lse2,
+                          float *lse_out, float *scores, int *status, bool first_pass, cudaStream_t stream)
 {
     constexpr int smem = Smem<D, STAGES>::kDynBytes;
     cudaError_t e = cudaFuncSetAttribute(importance_kernel<D, STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -385,7 +394,8 @@ cudaError_t launch_both(const CUtensorMap &mq, const CUtensorMap &mk, int units,
     e = cudaFuncSetAttribute(importance_kernel<D, STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)units * (unsigned)nt;
-    importance_kernel<D, STAGES, false><<<grid, kThreads, smem, stream>>>(mq, mk, T, nt, c, lse2, lse_out, scores, status);
+    if (first_pass)
+        importance_kernel<D, STAGES, false><<<grid, kThreads, smem, stream>>>(mq, mk, T, nt, c, lse2, lse_out, scores, status);
     importance_kernel<D, STAGES, true><<<grid, kThreads, smem, stream>>>(mq, mk, T, nt, c, lse2, lse_out, scores, status);
     return cudaGetLastError();
 }
@@ -399,7 +409,8 @@ size_t importance_workspace_bytes(int N, int H, int T, int D)
     return kStatusBytes + (size_t)N * H * nt * kTileRows * sizeof(float);   // status block + padded lse
 }
 
-cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out,
+// lse_in == nullptr: both passes. Otherwise the caller's normaliser replaces pass 1.
+cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out, const float *lse_in,
                               int N, int H, int T, int D, float scale, void *ws, cudaStream_t stream)
 {
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, stream);
@@ -408,12 +419,18 @@ cudaError_t launch_importance(const void *Q, const void *K, float *scores, float
     float *lse2 = reinterpret_cast<float *>(static_cast<char *>(ws) + kStatusBytes);
     const int units = N * H;
     const int nt = (T + kTileRows - 1) / kTileRows;
-    if ((long long)units * nt > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    if ((long long)units * nt > 0x7FFFFFFFLL || units > 65535 * 1024) return cudaErrorInvalidConfiguration;
     CUtensorMap mq, mk;
     if (!make_map(&mq, Q, units, T, D) || !make_map(&mk, K, units, T, D)) return cudaErrorInvalidValue;
+    if (lse_in) {
+        if (units > 65535) return cudaErrorInvalidConfiguration;
+        dim3 g((nt * kTileRows + 255) / 256, units);
+        lse_import_kernel<<<g, 256, 0, stream>>>(lse_in, lse2, T, nt * kTileRows);
+    }
     const float c = scale * kLog2e;
-    if (D == 128) return launch_both<128, 2>(mq, mk, units, T, nt, c, lse2, lse_out, scores, status, stream);
-    return launch_both<64, 4>(mq, mk, units, T, nt, c, lse2, lse_out, scores, status, stream);
+    if (D == 128)
+        return launch_passes<128, 2>(mq, mk, units, T, nt, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
+    return launch_passes<64, 4>(mq, mk, units, T, nt, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
 }
 
 }  // namespace ec

@@ -123,6 +123,29 @@ merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int
     }
 }
 
+// Eviction instead of merging: cache row k is the anchor's own row (everything else is dropped).
+// One lane group per kept row; grid.x = units * ceil(C / groups per CTA).
+template <int LPR>
+__global__ void __launch_bounds__(kMergeThreads)
+gather_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int32_t *__restrict__ anchor_pos,
+              int T, int C, int chunks, uint4 *__restrict__ Kc, uint4 *__restrict__ Vc, int cap)
+{
+    constexpr int GL = 2 * LPR;
+    constexpr int G = kMergeThreads / GL;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int unit = blockIdx.x / chunks;
+    const int chunk = blockIdx.x - unit * chunks;
+    const int g = threadIdx.x / GL, gl = threadIdx.x - g * GL;
+    const bool is_v = gl >= LPR;
+    const int l = is_v ? gl - LPR : gl;
+    const int k = chunk * G + g;
+    if (k >= C) return;
+    const int t = anchor_pos[(size_t)unit * C + k];
+    const uint4 *src = (is_v ? V : K) + ((size_t)unit * T + t) * LPR + l;
+    uint4 *dst = (is_v ? Vc : Kc) + ((size_t)unit * cap + k) * LPR + l;
+    *dst = ldg_stream(src);
+}
+
 template <int LPR>
 cudaError_t launch_merge_t(const void *K, const void *V, const int32_t *anchor_pos, unsigned grid, int T, int n_keep,
                            int slices, void *Kc, void *Vc, int cap, cudaStream_t stream)
@@ -146,6 +169,27 @@ cudaError_t launch_merge_t(const void *K, const void *V, const int32_t *anchor_p
                               (uint4 *)Kc, (uint4 *)Vc, cap);
 }
 
+template <int LPR>
+cudaError_t launch_gather_t(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int n_keep,
+                            void *Kc, void *Vc, int cap, cudaStream_t stream)
+{
+    constexpr int G = kMergeThreads / (2 * LPR);
+    const int chunks = (n_keep + G - 1) / G;
+    if ((long long)units * chunks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(units * chunks));
+    cfg.blockDim = dim3(kMergeThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gather_kernel<LPR>, (const uint4 *)K, (const uint4 *)V, anchor_pos, T, n_keep, chunks,
+                              (uint4 *)Kc, (uint4 *)Vc, cap);
+}
+
 }  // namespace
 
 cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
@@ -156,6 +200,13 @@ cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos
     if (grid > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     if (D == 128) return launch_merge_t<16>(K, V, anchor_pos, (unsigned)grid, T, n_keep, slices, Kc, Vc, cap, stream);
     return launch_merge_t<8>(K, V, anchor_pos, (unsigned)grid, T, n_keep, slices, Kc, Vc, cap, stream);
+}
+
+cudaError_t launch_gather(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
+                          int n_keep, void *Kc, void *Vc, int cap, cudaStream_t stream)
+{
+    if (D == 128) return launch_gather_t<16>(K, V, anchor_pos, units, T, n_keep, Kc, Vc, cap, stream);
+    return launch_gather_t<8>(K, V, anchor_pos, units, T, n_keep, Kc, Vc, cap, stream);
 }
 
 }  // namespace ec

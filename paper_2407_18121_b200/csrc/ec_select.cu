@@ -15,16 +15,17 @@ __device__ __forceinline__ uint32_t sort_key(float x)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Layer-wise population: mean over the heads of a problem. scores [N,H,T] -> mean [N,T].
-__global__ void head_mean_kernel(const float *__restrict__ scores, float *__restrict__ mean, int H, int T)
+// Shared population: mean over `share` consecutive units (the heads of a layer, or every
+// layer and head of a sequence). scores [G*share, T] -> mean [G, T].
+__global__ void group_mean_kernel(const float *__restrict__ scores, float *__restrict__ mean, int share, int T)
 {
-    int n = blockIdx.y;
-    int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t grp = blockIdx.y;
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
-    const float *s = scores + (size_t)n * H * T + t;
+    const float *s = scores + grp * share * T + t;
     float acc = 0.f;
-    for (int h = 0; h < H; ++h) acc += s[(size_t)h * T];
-    mean[(size_t)n * T + t] = acc / (float)H;
+    for (int j = 0; j < share; ++j) acc += s[(size_t)j * T];
+    mean[grp * T + t] = acc / (float)share;
 }
 
 // One CTA per selection unit. Dynamic shared memory: T keys + n_keep anchors.
@@ -145,21 +146,23 @@ select_kernel(const float *__restrict__ scores, int T, int C, int protect_ends, 
 
 }  // namespace
 
-cudaError_t launch_select(const float *scores, int N, int H, int T, int n_keep, int population,
-                          int protect_ends, int32_t *anchor_pos, int32_t *bucket_len, float *mean_ws,
-                          cudaStream_t stream)
+// `share` consecutive units rank one common (averaged) score vector; share == 1: every unit its own.
+cudaError_t launch_select(const float *scores, int units, int T, int n_keep, int share, int protect_ends,
+                          int32_t *anchor_pos, int32_t *bucket_len, float *mean_ws, cudaStream_t stream)
 {
     size_t smem = (size_t)(T + n_keep) * sizeof(uint32_t);
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    if (population == EC_LAYER_SHARED) {
-        dim3 g((T + 255) / 256, N);
-        head_mean_kernel<<<g, 256, 0, stream>>>(scores, mean_ws, H, T);
-        select_kernel<<<N, kSelThreads, smem, stream>>>(mean_ws, T, n_keep, protect_ends, H, anchor_pos, bucket_len);
+    if (share > 1) {
+        const int groups = units / share;
+        if (groups > 65535) return cudaErrorInvalidConfiguration;
+        dim3 g((T + 255) / 256, groups);
+        group_mean_kernel<<<g, 256, 0, stream>>>(scores, mean_ws, share, T);
+        select_kernel<<<groups, kSelThreads, smem, stream>>>(mean_ws, T, n_keep, protect_ends, share, anchor_pos, bucket_len);
     } else {
-        select_kernel<<<N * H, kSelThreads, smem, stream>>>(scores, T, n_keep, protect_ends, 1, anchor_pos, bucket_len);
+        select_kernel<<<units, kSelThreads, smem, stream>>>(scores, T, n_keep, protect_ends, 1, anchor_pos, bucket_len);
     }
     return cudaGetLastError();
 }

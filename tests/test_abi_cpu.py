@@ -93,3 +93,16 @@ def test_cache_init_and_decode_validation(L):
     assert step(p, p, p, C.byref(c), 1.0, p, C.byref(ev), None, None, 0, None) == 5
     assert (c.len, c.ring_head, c.step) == (8, 0, 0)               # failed calls leave the state alone
     assert L.ec_decode_workspace(C.byref(c)) >= 256
+
+
+def test_ratio_cache_init_validation(L):
+    p = 0x10000
+    c = ec.ec_cache()
+    ring = (C.c_int * 8)()
+    f = L.ec_cache_init_ratio
+    assert f(C.byref(c), p, p, 1, 2, 64, 64, 20, 8, 0.5, 40, ring) == 0
+    assert list(ring) == list(range(12, 20)) and c.policy == 1 and c.n_tot == 40 and c.len == 20
+    assert f(C.byref(c), p, p, 1, 2, 64, 64, 20, 8, 0.5, 40, None) == 1       # ring missing
+    assert f(C.byref(c), p, p, 1, 2, 64, 64, 6, 8, 0.5, 40, ring) == 4        # fewer rows than the offset
+    assert f(C.byref(c), p, p, 1, 2, 64, 64, 20, 8, 0.0, 40, ring) == 4       # ratio out of range
+    assert f(C.byref(c), p, p, 1, 2, 64, 64, 20, 8, 0.5, 10, ring) == 4       # fewer tokens seen than rows held

@@ -327,3 +327,20 @@ def test_ratio_policy_follows_algorithm_1_count():
             assert pos == -1
         assert qd.len == length
         assert length <= n_tot * ratio + 1
+
+
+# ------------------------------------------------------------------ ablation variants
+
+def test_group_mean_and_gather_reduce_to_numpy():
+    rng = np.random.default_rng(31)
+    s = rng.random((12, 17))
+    np.testing.assert_allclose(orc.group_mean(s, 4), s.reshape(3, 4, 17).mean(1), rtol=1e-14)
+    np.testing.assert_allclose(orc.group_mean(s, 1), s, rtol=0)
+    np.testing.assert_allclose(orc.group_mean(s, 12)[0], s.mean(0), rtol=1e-14)
+    np.testing.assert_allclose(orc.group_mean(s, 4), orc.layer_mean(s.reshape(3, 4, 17)), rtol=1e-15)
+    Xb = _rand_bits(rng, (2, 9, 4))
+    a = np.array([[0, 3, 8], [1, 2, 7]], np.int32)
+    got = orc.gather(Xb, a)
+    X = wl.bf16_bits_to_f64(Xb)
+    for u in range(2):
+        np.testing.assert_array_equal(got[u], X[u, a[u]])

@@ -360,3 +360,106 @@ def test_whole_path_on_workload(name, population):
         assert ev == (C - w.offset) + (s % w.offset) and pos == C - w.offset
         assert_bf16_close(out, want, f"decode out, step {s}")
     assert cache.len == C
+
+
+# ---------------------------------------------------------------- retention-ratio policy
+
+@pytest.mark.parametrize("T,ratio,offset,steps,N,H,D", [(200, 0.3, 16, 150, 2, 3, 128), (90, 0.5, 25, 80, 1, 8, 64),
+                                                        (64, 1.0, 4, 20, 1, 2, 128)])
+def test_decode_ratio_policy_grows_and_evicts_like_the_oracle(T, ratio, offset, steps, N, H, D):
+    """The budget follows keep_ratio x tokens seen: some steps append, some evict at the fixed
+    truncation location. Same rows must leave on both sides, and outputs must agree."""
+    rng = np.random.default_rng(T)
+    C = orc.keep_count(T, ratio)
+    cap = C + steps
+    K0b, V0b = rand_bits(rng, (N, H, C, D)), rand_bits(rng, (N, H, C, D))
+    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=cap + 1)
+    Kc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
+    Vc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
+    Kc.t[:, :, :C] = dev_bf16(K0b)
+    Vc.t[:, :, :C] = dev_bf16(V0b)
+    cache = ec.ec_cache_init_ratio(Kc.t, Vc.t, C, offset, ratio, T)
+    ws = scratch(ec.ec_decode_workspace(cache))
+    slot_ids = list(range(C)) + [-1] * (cap - C)
+    grew = evicted_n = 0
+    for s in range(steps):
+        qb, kb, vb = rand_bits(rng, (N, H, D)), rand_bits(rng, (N, H, D)), rand_bits(rng, (N, H, D))
+        len_before = cache.len
+        want, pos, ident = queue.step(qb, kb, vb, 0.1, policy=orc.POLICY_RATIO, offset=offset, ratio=ratio,
+                                      n_tot=T + s + 1)
+        out = torch.empty((N, H, D), dtype=torch.bfloat16, device="cuda")
+        ev, slot = ec.ec_decode_step(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), cache, 0.1, out, ws)
+        assert_bf16_close(out, want, f"decode out, step {s}")
+        if pos < 0:
+            assert ev == -1 and slot == len_before and cache.len == len_before + 1
+            grew += 1
+        else:
+            assert pos == len_before - offset and ev == slot and slot_ids[ev] == ident and cache.len == len_before
+            evicted_n += 1
+        slot_ids[slot] = queue.next_id - 1
+        assert cache.len == queue.len and cache.n_tot == T + s + 1
+        assert sorted(slot_ids[:cache.len]) == sorted(queue.identities().tolist())
+    assert grew > 0 and (evicted_n > 0 or ratio == 1.0)
+    Kc.check("Kc")
+    Vc.check("Vc")
+    Kdev = host_f64(Kc.t[:, :, :cache.len])
+    for j, ident in enumerate(queue.identities().tolist()):
+        np.testing.assert_array_equal(Kdev[:, :, slot_ids.index(ident)], queue.K[:, j].reshape(N, H, D))
+
+
+# ---------------------------------------------------------------- importance from a given normaliser
+
+@pytest.mark.parametrize("N,H,T,D", [(1, 2, 129, 128), (2, 2, 300, 64), (1, 3, 640, 128)])
+def test_importance_from_lse_matches_oracle(N, H, T, D):
+    rng = np.random.default_rng(T + 11)
+    Qb, Kb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    scale = 1.0 / math.sqrt(D)
+    want, o_lse = orc.importance(Qb, Kb, scale)
+    lse = torch.from_numpy(o_lse.astype(np.float32)).cuda()       # the oracle's normaliser as the input
+    scores = Guarded((N, H, T), torch.float32, fill=float("nan"))
+    ws = scratch(ec.ec_importance_workspace(N, H, T, D))
+    ec.ec_importance_from_lse(dev_bf16(Qb), dev_bf16(Kb), lse, scores.t, scale, ws)
+    assert ec.ec_device_status(ws) == ec.EC_OK
+    scores.check("scores")
+    assert_rel_close(scores.t, want, SCORE_RTOL, what="scores from lse")
+
+
+# ---------------------------------------------------------------- ablation variants of the compaction
+
+def gpu_select_compact(Kb, Vb, s32, n_keep, share, protect, compaction):
+    N, H, T, D = Kb.shape
+    Kc = Guarded((N, H, n_keep, D), torch.bfloat16, fill=float("nan"))
+    Vc = Guarded((N, H, n_keep, D), torch.bfloat16, fill=float("nan"))
+    anchors = Guarded((N, H, n_keep), torch.int32, fill=-7)
+    ws = scratch(ec.ec_select_compact_workspace(N, H, T, D, n_keep, share))
+    ec.ec_select_compact(dev_bf16(Kb), dev_bf16(Vb), torch.from_numpy(s32).cuda(), n_keep, share, protect, compaction,
+                         Kc.t, Vc.t, anchors.t, None, ws)
+    for g, name in ((Kc, "Kc"), (Vc, "Vc"), (anchors, "anchor_pos")):
+        g.check(name)
+    return Kc.t, Vc.t, anchors.t
+
+
+@pytest.mark.parametrize("share_kind", ["head", "layer", "sequence"])
+@pytest.mark.parametrize("compaction", [ec.EC_COMPACT_MERGE, ec.EC_COMPACT_EVICT])
+def test_select_compact_populations_and_eviction(share_kind, compaction):
+    B, Lyr, H, T, D, n_keep = 2, 3, 4, 260, 128, 40
+    N = B * Lyr
+    share = {"head": 1, "layer": H, "sequence": Lyr * H}[share_kind]
+    rng = np.random.default_rng(share + compaction)
+    Kb, Vb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    s32 = (rng.random((N, H, T)) ** 3 + 1e-3).astype(np.float32)
+    s64 = s32.astype(np.float64).reshape(N * H, T)
+    rank = np.repeat(orc.group_mean(s64, share), share, axis=0).reshape(N, H, T)
+    want_anchors = orc.select(rank, n_keep, True)
+    Kc, Vc, anchors = gpu_select_compact(Kb, Vb, s32, n_keep, share, True, compaction)
+    check_anchor_sets(anchors, want_anchors, rank, n_keep, True)
+    ga = anchors.cpu().numpy().reshape(N * H // share, share, n_keep)
+    assert (ga == ga[:, :1]).all()                               # one anchor set per sharing group
+    use = anchors_to_merge_on(anchors, want_anchors)
+    if compaction == ec.EC_COMPACT_EVICT:
+        np.testing.assert_array_equal(host_f64(Kc), orc.gather(Kb, use))     # copies: bit-exact
+        np.testing.assert_array_equal(host_f64(Vc), orc.gather(Vb, use))
+    else:
+        lo, hi = orc.buckets(use, T)
+        assert_bf16_close(Kc, orc.merge(Kb, lo, hi), "merged K")
+        assert_bf16_close(Vc, orc.merge(Vb, lo, hi), "merged V")
