@@ -200,8 +200,15 @@ size_t ec_decode_workspace(const ec_cache *c)
     return 256 + round256((size_t)units * splits * (c->D + 2) * sizeof(float));
 }
 
-int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
-                   int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream)
+}  // extern "C"
+
+namespace {
+
+// One decode step. `prev_slot` >= 0 promises that the kernel enqueued on `stream` right before
+// this call is the decode step that stored cache row `prev_slot` and nothing else this step
+// reads; the kernel may then read the rest of the cache while that step is still finishing.
+int decode_step_impl(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
+                     int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream, int prev_slot)
 {
     if (!q || !k_new || !v_new || !c || !out || !evicted_slot) return EC_ERR_NULL;
     if (!c->Kc || !c->Vc) return EC_ERR_NULL;
@@ -245,8 +252,8 @@ int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache
     const int units = c->N * c->H;
     const int splits = ec::decode_splits(units, c->len + 1);
     float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
-    cudaError_t e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, scale,
-                                      out, partials, splits, (cudaStream_t)stream);
+    cudaError_t e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, prev_slot,
+                                      scale, out, partials, splits, (cudaStream_t)stream);
     if (e != cudaSuccess) return EC_ERR_CUDA;
     if (ratio) {
         // the new row is now the newest; the ring's oldest entry either left or stops being tracked
@@ -265,19 +272,31 @@ int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache
     return EC_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
+                   int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream)
+{
+    return decode_step_impl(q, k_new, v_new, c, scale, out, evicted_slot, slot_written, ws, ws_bytes, stream, -1);
+}
+
 int ec_decode_steps(const void *q, const void *k_new, const void *v_new, int steps, ec_cache *c, float scale,
                     void *out, int *evicted_slots, void *ws, size_t ws_bytes, void *stream)
 {
     if (steps < 0) return EC_ERR_ARG;
     if (!c) return EC_ERR_NULL;
     const size_t stride = (size_t)c->N * c->H * c->D * 2;   // bytes of one [N, H, D] bf16 step
+    int prev = -1;       // the first step of the call knows nothing about the kernel before it
     for (int s = 0; s < steps; ++s) {
-        int ev = -1;
-        int st = ec_decode_step(static_cast<const char *>(q) + s * stride, static_cast<const char *>(k_new) + s * stride,
-                                static_cast<const char *>(v_new) + s * stride, c, scale,
-                                static_cast<char *>(out) + s * stride, &ev, nullptr, ws, ws_bytes, stream);
+        int ev = -1, slot = -1;
+        int st = decode_step_impl(static_cast<const char *>(q) + s * stride, static_cast<const char *>(k_new) + s * stride,
+                                  static_cast<const char *>(v_new) + s * stride, c, scale,
+                                  static_cast<char *>(out) + s * stride, &ev, &slot, ws, ws_bytes, stream, prev);
         if (st != EC_OK) return st;
         if (evicted_slots) evicted_slots[s] = ev;
+        prev = slot;
     }
     return EC_OK;
 }

@@ -69,7 +69,7 @@ cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos
 
 int decode_splits(int units, int rows);
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
-                          int units, int D, int cap, int len, int write_slot, float scale, void *out,
+                          int units, int D, int cap, int len, int write_slot, int defer_row, float scale, void *out,
                           float *partials, int splits, cudaStream_t stream);
 
 }  // namespace ec

@@ -129,7 +129,7 @@ __device__ __forceinline__ void process_block(GroupState &st, const float2 (&q2)
 template <int LPR>
 __global__ void __launch_bounds__(kDecThreads, EC_DEC_MIN_CTAS)
 decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-              uint4 *Kc, uint4 *Vc, int cap, int len, int write_slot, float scale_log2e,
+              uint4 *Kc, uint4 *Vc, int cap, int len, int write_slot, int defer_row, float scale_log2e,
               __nv_bfloat16 *__restrict__ out, float *__restrict__ partials, int splits)
 {
     constexpr int D = LPR * 8;
@@ -137,11 +137,16 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
     __shared__ float sm_acc[G][D];
     __shared__ float sm_m[G], sm_l[G];
 
-    // Launched with programmatic stream serialization: nothing in global memory is touched
-    // before the previous kernel of the stream has completed; the next launch may then start
-    // scheduling its CTAs while this one runs.
-    grid_dependency_wait();
-    grid_launch_dependents();
+    // Launched with programmatic stream serialization. defer_row < 0: nothing in global memory
+    // is touched before the previous kernel of the stream has completed. defer_row >= 0: the
+    // previous kernel is the decode step before this one, which changes nothing this step reads
+    // except cache row `defer_row` (the row it stored); everything else is read first, and only
+    // the block holding that row, and every write, wait for the predecessor. The next launch is
+    // released only after that wait, so at most two consecutive steps ever overlap.
+    if (defer_row < 0) {
+        grid_dependency_wait();
+        grid_launch_dependents();
+    }
 
     const int unit = blockIdx.x / splits;
     const int split = blockIdx.x - unit * splits;
@@ -176,9 +181,20 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
     for (int i = 0; i < 4; ++i) st.acc[i] = make_float2(0.f, 0.f);
 
     const uint4 *Kl = Kcu + l, *Vl = Vcu + l;
-    for (int b = g; b < nfull; b += G) process_block<LPR, false>(st, q2, Kl, Vl, r0 + b * kBlk, r1, l, gmask);
-    if (r0 + nfull * kBlk < r1 && (nfull % G) == g)
+    const bool has_tail = r0 + nfull * kBlk < r1;
+    const int bd = (defer_row >= r0 && defer_row < r1) ? (defer_row - r0) / kBlk : -1;   // block put off
+    for (int b = g; b < nfull; b += G)
+        if (b != bd) process_block<LPR, false>(st, q2, Kl, Vl, r0 + b * kBlk, r1, l, gmask);
+    if (has_tail && (nfull % G) == g && bd != nfull)
         process_block<LPR, true>(st, q2, Kl, Vl, r0 + nfull * kBlk, r1, l, gmask);
+    if (defer_row >= 0) {
+        grid_dependency_wait();
+        grid_launch_dependents();
+        if (bd >= 0 && (bd % G) == g) {
+            if (bd < nfull) process_block<LPR, false>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
+            else            process_block<LPR, true>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
+        }
+    }
 
     // per-lane partial sums -> group sum (rows are owned by LPR/8 lanes each)
     float lsum = st.lsum;
@@ -303,12 +319,13 @@ cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, unsigned 
 
 template <int LPR>
 cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc, int units,
-                            int cap, int len, int write_slot, float sl2, void *out, float *partials, int splits,
-                            cudaStream_t stream)
+                            int cap, int len, int write_slot, int defer_row, float sl2, void *out, float *partials,
+                            int splits, cudaStream_t stream)
 {
     cudaError_t e = launch_overlapped(decode_kernel<LPR>, (unsigned)(units * splits), (unsigned)kDecThreads, stream,
                                       (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc,
-                                      (uint4 *)Vc, cap, len, write_slot, sl2, (__nv_bfloat16 *)out, partials, splits);
+                                      (uint4 *)Vc, cap, len, write_slot, splits == 1 ? defer_row : -1, sl2, (__nv_bfloat16 *)out,
+                                      partials, splits);
     if (e != cudaSuccess || splits == 1) return e;
     return launch_overlapped(combine_kernel<LPR>, (unsigned)units, (unsigned)(LPR * 8), stream,
                              (const float *)partials, splits, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc,
@@ -316,14 +333,14 @@ cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new,
 }
 
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
-                          int units, int D, int cap, int len, int write_slot, float scale, void *out,
+                          int units, int D, int cap, int len, int write_slot, int defer_row, float scale, void *out,
                           float *partials, int splits, cudaStream_t stream)
 {
     const float sl2 = scale * 1.4426950408889634f;
     if ((long long)units * splits > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     if (D == 128)
-        return launch_decode_t<16>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, sl2, out, partials, splits, stream);
-    return launch_decode_t<8>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, sl2, out, partials, splits, stream);
+        return launch_decode_t<16>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials, splits, stream);
+    return launch_decode_t<8>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials, splits, stream);
 }
 
 }  // namespace ec

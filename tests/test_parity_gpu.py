@@ -463,3 +463,36 @@ def test_select_compact_populations_and_eviction(share_kind, compaction):
         lo, hi = orc.buckets(use, T)
         assert_bf16_close(Kc, orc.merge(Kb, lo, hi), "merged K")
         assert_bf16_close(Vc, orc.merge(Vb, lo, hi), "merged V")
+
+
+def test_decode_steps_overlapped_loop_with_many_units():
+    """With enough units for one CTA per unit, the native loop lets step s+1 read the cache while
+    step s is still finishing, putting off only the row step s stores. Rows stored by earlier steps
+    sit in full blocks and in the ragged last block here; results must match the one-step calls
+    and the oracle."""
+    rng = np.random.default_rng(12)
+    N, H, D, C, d, S = 20, 32, 128, 45, 10, 33
+    K0b, V0b = rand_bits(rng, (N, H, C, D)), rand_bits(rng, (N, H, C, D))
+    qb, kb, vb = (rand_bits(rng, (S, N, H, D)) for _ in range(3))
+    K0, V0 = dev_bf16(K0b), dev_bf16(V0b)
+    q, k, v = dev_bf16(qb), dev_bf16(kb), dev_bf16(vb)
+    Ka, Va, Kb_, Vb_ = K0.clone(), V0.clone(), K0.clone(), V0.clone()
+    ca, cb = ec.ec_cache_init(Ka, Va, C, C, d), ec.ec_cache_init(Kb_, Vb_, C, C, d)
+    ws = scratch(ec.ec_decode_workspace(ca))
+    out_a = torch.empty((S, N, H, D), dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty_like(out_a)
+    for s in range(S):
+        ec.ec_decode_step(q[s], k[s], v[s], ca, 0.09, out_a[s], ws)
+    slots = ec.ec_decode_steps(q, k, v, cb, 0.09, out_b, ws, want_slots=True)
+    torch.cuda.synchronize()
+    assert slots == [(C - d) + (s % d) for s in range(S)]
+    assert torch.equal(Ka, Kb_) and torch.equal(Va, Vb_)
+    a, b = host_f64(out_a), host_f64(out_b)
+    assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(a) + 1e-6).all()          # same result up to block order
+    for (n, h) in [(0, 0), (7, 13), (19, 31)]:
+        queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b[n, h][None]), wl.bf16_bits_to_f64(V0b[n, h][None]), cap=C + 1)
+        for s in range(S):
+            want, _, _ = queue.step(qb[s, n, h][None], kb[s, n, h][None], vb[s, n, h][None], 0.09,
+                                    policy=orc.POLICY_FIXED, budget=C, offset=d)
+            err = np.abs(b[s, n, h] - want[0])
+            assert (err <= 2e-2 + 2.0 ** -8 * np.abs(want[0])).all(), (n, h, s)
