@@ -86,6 +86,24 @@ int ec_importance(const void *Q_dev, const void *K_dev, float *scores_dev, float
                   void *ws_dev, size_t ws_bytes, void *stream);
 
 /*
+ * Importance when a new instruction of Tq tokens is encoded on top of P rows that are already
+ * in the cache (Sec. 3.1: the instruction stage also takes in chat history; Eq. 1 with the
+ * queries being the last Tq tokens): query m sees keys n <= m + P, and
+ *   scores[n] = sum over the Tq queries of A[m][n],  n = 0 .. P+Tq-1.
+ * The caller concatenates the cached rows and the new rows (K and, for ec_select_merge, V)
+ * and compacts the P+Tq rows as usual. P = 0 is ec_importance.
+ *   Q_dev       bf16 [N, H, Tq, D]                                   (in)
+ *   K_dev       bf16 [N, H, P+Tq, D]                                 (in)
+ *   scores_dev  fp32 [N, H, P+Tq]                                    (out)
+ *   lse_dev     fp32 [N, H, Tq], natural log; may be NULL            (out, optional)
+ *   ws_dev      scratch of ec_importance_workspace(N, H, Tq, D) bytes
+ * Limits: Tq >= 1, P >= 0, P + Tq <= 16384.
+ */
+int ec_importance_prefix(const void *Q_dev, const void *K_dev, float *scores_dev, float *lse_dev,
+                         int N, int H, int Tq, int P, int D, float scale,
+                         void *ws_dev, size_t ws_bytes, void *stream);
+
+/*
  * The same importance when the caller already holds every query row's log-sum-exp, as a
  * prefill attention kernel produces it (the paper takes the attention probabilities from
  * the model's own forward pass, Algorithm 1 "Input"): only the column-sum pass runs, which

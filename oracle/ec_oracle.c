@@ -128,6 +128,46 @@ void eco_importance(const uint16_t *Q, const uint16_t *K, int U, int T, int D, d
     }
 }
 
+/*
+ * The same definition when the queries are only the LAST Tq tokens of a sequence of P + Tq keys
+ * (a new instruction encoded on top of P rows that are already in the cache, Sec. 3.1: the
+ * instruction stage also covers chat history): query m sees keys n <= m + P, and
+ * I[n] = sum over the Tq queries of A[m][n]. P = 0 is eco_importance.
+ * Q: bf16 [U, Tq, D]; K: bf16 [U, P+Tq, D]; scores [U, P+Tq]; lse (nullable) [U, Tq].
+ */
+void eco_importance_prefix(const uint16_t *Q, const uint16_t *K, int U, int Tq, int P, int D, double scale,
+                           double *scores, double *lse)
+{
+    const int Tk = P + Tq;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < U; ++u) {
+        double *q = (double *)malloc(sizeof(double) * (size_t)Tq * D);
+        double *k = (double *)malloc(sizeof(double) * (size_t)Tk * D);
+        double *s = (double *)malloc(sizeof(double) * (size_t)Tk);
+        eco_widen_bf16(Q + (size_t)u * Tq * D, (int64_t)Tq * D, q);
+        eco_widen_bf16(K + (size_t)u * Tk * D, (int64_t)Tk * D, k);
+        double *I = scores + (size_t)u * Tk;
+        for (int n = 0; n < Tk; ++n) I[n] = 0.0;
+        for (int m = 0; m < Tq; ++m) {
+            const int last = m + P;
+            double mx = -INFINITY;
+            for (int n = 0; n <= last; ++n) {
+                double dot = 0.0;
+                for (int c = 0; c < D; ++c) dot += q[(size_t)m * D + c] * k[(size_t)n * D + c];
+                s[n] = scale * dot;
+                if (s[n] > mx) mx = s[n];
+            }
+            double Z = 0.0;
+            for (int n = 0; n <= last; ++n) Z += exp(s[n] - mx);
+            for (int n = 0; n <= last; ++n) I[n] += exp(s[n] - mx) / Z;
+            if (lse) lse[(size_t)u * Tq + m] = mx + log(Z);
+        }
+        free(q);
+        free(k);
+        free(s);
+    }
+}
+
 /* Layer-wise population: the mean over the heads of a layer. scores [N, H, T] -> out [N, T]. */
 void eco_layer_mean(const double *scores, int N, int H, int T, double *out)
 {

@@ -28,6 +28,8 @@ _lib.eco_keep_count.restype = C.c_int
 _lib.eco_keep_count.argtypes = [C.c_int, C.c_double]
 _lib.eco_importance.restype = None
 _lib.eco_importance.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_double, _f64p, _f64p]
+_lib.eco_importance_prefix.restype = None
+_lib.eco_importance_prefix.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _f64p, _f64p]
 _lib.eco_layer_mean.restype = None
 _lib.eco_layer_mean.argtypes = [_f64p, C.c_int, C.c_int, C.c_int, _f64p]
 _lib.eco_group_mean.restype = None
@@ -78,6 +80,20 @@ def importance(Q: np.ndarray, K: np.ndarray, scale: float) -> Tuple[np.ndarray, 
     scores = np.empty(Q.shape[:-1], np.float64)
     lse = np.empty(Q.shape[:-1], np.float64)
     _lib.eco_importance(_p(Q, _u16p), _p(K, _u16p), U, T, D, float(scale), _p(scores, _f64p), _p(lse, _f64p))
+    return scores, lse
+
+
+def importance_prefix(Q: np.ndarray, K: np.ndarray, scale: float) -> Tuple[np.ndarray, np.ndarray]:
+    """Q uint16 [..., Tq, D], K uint16 [..., P+Tq, D] (P >= 0 earlier keys every query sees).
+    Returns (scores [..., P+Tq], lse [..., Tq]) in float64."""
+    Q, K = _bits(Q), _bits(K)
+    assert Q.shape[:-2] == K.shape[:-2] and Q.shape[-1] == K.shape[-1] and K.shape[-2] >= Q.shape[-2]
+    Tq, D = Q.shape[-2:]
+    P = K.shape[-2] - Tq
+    U = int(np.prod(Q.shape[:-2], dtype=np.int64))
+    scores = np.empty(K.shape[:-1], np.float64)
+    lse = np.empty(Q.shape[:-1], np.float64)
+    _lib.eco_importance_prefix(_p(Q, _u16p), _p(K, _u16p), U, Tq, P, D, float(scale), _p(scores, _f64p), _p(lse, _f64p))
     return scores, lse
 
 

@@ -22,7 +22,7 @@ EC_LAYER_SHARED = 1
 
 EXPORTS = (
     "ec_status_string", "ec_keep_count",
-    "ec_importance_workspace", "ec_importance", "ec_importance_from_lse", "ec_device_status",
+    "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_from_lse", "ec_device_status",
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
     "ec_cache_init", "ec_cache_init_ratio", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc",
@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
     L.ec_importance_workspace.argtypes = [i, i, i, i]
     L.ec_importance.restype = i
     L.ec_importance.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
+    L.ec_importance_prefix.restype = i
+    L.ec_importance_prefix.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
     L.ec_importance_from_lse.restype = i
     L.ec_importance_from_lse.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
     L.ec_device_status.restype = i
@@ -135,6 +137,17 @@ def ec_importance(Q: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, lse: O
     st = lib().ec_importance(_ptr(Q), _ptr(K), _ptr(scores), _ptr(lse), N, H, T, D, float(scale),
                              _ptr(ws), ws.numel() * ws.element_size(), _stream())
     _check(st, "ec_importance")
+
+
+def ec_importance_prefix(Q: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, lse: Optional[torch.Tensor],
+                         scale: float, ws: torch.Tensor) -> None:
+    """Q: bf16 [N,H,Tq,D]; K: bf16 [N,H,P+Tq,D] (P earlier rows every query sees); scores (out): fp32
+    [N,H,P+Tq]; lse (out, optional): fp32 [N,H,Tq]; ws sized by ec_importance_workspace(N,H,Tq,D)."""
+    N, H, Tq, D = Q.shape
+    P = K.shape[2] - Tq
+    st = lib().ec_importance_prefix(_ptr(Q), _ptr(K), _ptr(scores), _ptr(lse), N, H, Tq, P, D, float(scale),
+                                    _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_importance_prefix")
 
 
 def ec_importance_from_lse(Q: torch.Tensor, K: torch.Tensor, lse: torch.Tensor, scores: torch.Tensor,

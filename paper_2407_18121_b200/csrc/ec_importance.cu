@@ -1,15 +1,20 @@
 // Importance of every prompt key (Sec. 3.3, Eq. 1 and the column sums that follow it),
-// computed in two passes so that the T x T attention matrix is never stored:
-//   pass 1: lse[m]   = log2 sum_{n<=m} 2^(c*<q_m,k_n>)          c = scale*log2(e)
-//   pass 2: score[n] = sum_{m>=n} 2^(c*<q_m,k_n> - lse[m])
+// computed in two passes so that the attention matrix is never stored:
+//   pass 1: lse[m]   = log2 sum_{n<=m+P} 2^(c*<q_m,k_n>)          c = scale*log2(e)
+//   pass 2: score[n] = sum_{m>=n-P} 2^(c*<q_m,k_n> - lse[m])
+// P is the number of keys that precede the first query (0 for a plain prompt; the rows of
+// an earlier, already compacted cache when a new instruction is encoded on top of it).
 // Both passes are the same dense causal contraction, run on the 5th-generation tensor
 // cores: 128x128 score tiles are produced by tcgen05.mma from TMA-staged bf16 tiles into
 // TMEM, and read back one row per thread, so a thread owns a query row in pass 1 and a key
 // row in pass 2 and every reduction stays inside a thread (no atomics, run-to-run identical).
 //
-// One CTA owns a "stationary" 128-row tile of one unit and streams the other operand's tiles
-// past it. Warp roles: warp 0 issues TMA loads, warp 1 issues MMAs and owns the TMEM
-// allocation, warps 2..5 (one thread per TMEM lane) do the softmax arithmetic.
+// A work item is a "stationary" 128-row tile of one unit, past which the other operand's
+// tiles are streamed. CTAs are persistent (two per SM): each walks a fixed list of item
+// pairs (a heavy tile and its light complement, so that pairs cost about the same) and
+// keeps its barriers, TMEM allocation and TMA ring alive across items. Warp roles: warp 0
+// issues TMA loads, warp 1 issues MMAs and owns the TMEM allocation, warps 2..5 (one thread
+// per TMEM lane) do the softmax arithmetic.
 // Every mbarrier wait is bounded in time; on expiry the CTA records a status word and leaves.
 #include "ec_common.cuh"
 
@@ -111,10 +116,9 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+// 32 consecutive fp32 columns of this thread's TMEM lane; the data is valid after tmem_ld_wait.
+__device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t (&r)[32])
 {
-    uint32_t r[32];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                  "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
                  "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
@@ -123,9 +127,52 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
                    "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr));
+}
+
+// Waits for every outstanding TMEM load of this thread; the registers of `r` are marked as
+// redefined here so that no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32])
+{
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 32; ++i) asm volatile("" : "+r"(r[i]));
+}
+
+// 2^x on the FMA pipe (Cody-Waite split + degree-4 polynomial, relative error < 6e-6) for
+// x <= ~0. One element in EC_IMP_POLY_EVERY goes this way, to take some load off the
+// special-function unit (one ex2 per score element is the busiest pipe of these kernels).
+#ifndef EC_IMP_POLY_EVERY
+#define EC_IMP_POLY_EVERY 4          // 0 = never
+#endif
+__device__ __forceinline__ float poly_exp2(float x)
+{
+    x = fmaxf(x, -125.f);                               // below this the result is ~0 anyway
+    const float t = x + 12582912.f;                     // 1.5 * 2^23: the low mantissa bits now hold round(x)
+    const float f = x - (t - 12582912.f);               // fractional part in [-0.5, 0.5]
+    float p = fmaf(f, 0.00935919489711523f, 0.05588679388165474f);
+    p = fmaf(p, f, 0.2402936965227127f);
+    p = fmaf(p, f, 0.6931265592575073f);
+    p = fmaf(p, f, 0.9999980926513672f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));   // scale by 2^round(x)
+}
+
+template <int I>
+__device__ __forceinline__ float exp2_mixed(float x)
+{
+    constexpr int every = EC_IMP_POLY_EVERY > 0 ? EC_IMP_POLY_EVERY : 1;
+    if (EC_IMP_POLY_EVERY > 0 && (I % every) == every - 1) return poly_exp2(x);
+    return fast_exp2(x);
+}
+
+// part[i & 3] += 2^(v[i]*c - m) over the 32 values of a chunk, unrolled at compile time so that
+// the choice between ex2 and the polynomial is static per element.
+template <int I>
+__device__ __forceinline__ void sum_exp2(const float (&v)[32], float c, float m, float (&part)[4])
+{
+    if constexpr (I < 32) {
+        part[I & 3] += exp2_mixed<I>(fmaf(v[I], c, -m));
+        sum_exp2<I + 1>(v, c, m, part);
+    }
 }
 
 template <int D, int STAGES>
@@ -135,23 +182,33 @@ struct Smem {
     static constexpr int kStage0 = kTileBytes;
     static constexpr int kLse = kStage0 + STAGES * kTileBytes;            // 2 x 128 floats
     static constexpr int kBars = kLse + kAccBufs * kTileRows * 4;
-    // barrier slots (8 bytes each): stat_full, full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], lse_ready[2]
-    static constexpr int kNumBars = 1 + 2 * STAGES + 3 * kAccBufs;
+    // barrier slots (8 bytes each): stat_full, stat_empty, full[STAGES], empty[STAGES],
+    // acc_full[2], acc_empty[2], lse_ready[2]
+    static constexpr int kNumBars = 2 + 2 * STAGES + 3 * kAccBufs;
     static constexpr int kTmemSlot = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemSlot + 4;
     static constexpr int kTotal = kAbort + 4;
     static constexpr int kDynBytes = kTotal + 1024;                       // slack for 1024-byte alignment
 };
 
-// PASS2 == false: stationary = query tile i, streamed = key tiles i, i-1, .., 0   -> lse2 (and lse_out)
-// PASS2 == true : stationary = key tile j,   streamed = query tiles j, j+1, .., nt-1 -> scores
-// The first streamed tile is always the diagonal one (the only tile that needs the causal mask).
-// lse2 is padded to nt*128 entries per unit; entries past T hold +inf so that pass 2 gives
-// those (non-existent) queries zero weight.
+// Geometry of the causal contraction with a visible prefix: query m sees keys n <= m + P.
+struct Geometry {
+    int Tq, P, ntq, ntk;
+    __host__ __device__ int Tk() const { return Tq + P; }
+    // pass 1: last key tile a query tile touches
+    __host__ __device__ int jmax(int i) const { int j = (i * kTileRows + kTileRows - 1 + P) / kTileRows; return j < ntk - 1 ? j : ntk - 1; }
+    // pass 2: first query tile that sees a key tile
+    __host__ __device__ int imin(int j) const { int d = j * kTileRows - P; return d > 0 ? d / kTileRows : 0; }
+};
+
+// PASS2 == false: stationary = query tile i, streamed = key tiles jmax(i) .. 0      -> lse2 (and lse_out)
+// PASS2 == true : stationary = key tile j,   streamed = query tiles imin(j) .. ntq-1 -> scores
+// A streamed tile needs the mask only when 128*(i-j) + P < 127. lse2 is padded to ntq*128 entries
+// per unit; entries past Tq hold +inf so that pass 2 gives those (non-existent) queries zero weight.
 template <int D, int STAGES, bool PASS2>
 __global__ void __launch_bounds__(kThreads, 2)
 importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  int T, int nt, float c, float *__restrict__ lse2, float *__restrict__ lse_out,
+                  const Geometry geo, int n_super, float c, float *__restrict__ lse2, float *__restrict__ lse_out,
                   float *__restrict__ scores, int *__restrict__ status)
 {
     using L = Smem<D, STAGES>;
@@ -164,23 +221,21 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bars = base + L::kBars;
-    const uint32_t bar_stat = bars;
-    auto bar_full = [&](int s) { return bars + 8u * (1 + s); };
-    auto bar_empty = [&](int s) { return bars + 8u * (1 + STAGES + s); };
-    auto bar_acc_full = [&](int b) { return bars + 8u * (1 + 2 * STAGES + b); };
-    auto bar_acc_empty = [&](int b) { return bars + 8u * (1 + 2 * STAGES + kAccBufs + b); };
-    auto bar_lse = [&](int b) { return bars + 8u * (1 + 2 * STAGES + 2 * kAccBufs + b); };
+    const uint32_t bar_stat_full = bars, bar_stat_empty = bars + 8u;
+    auto bar_full = [&](int s) { return bars + 8u * (2 + s); };
+    auto bar_empty = [&](int s) { return bars + 8u * (2 + STAGES + s); };
+    auto bar_acc_full = [&](int b) { return bars + 8u * (2 + 2 * STAGES + b); };
+    auto bar_acc_empty = [&](int b) { return bars + 8u * (2 + 2 * STAGES + kAccBufs + b); };
+    auto bar_lse = [&](int b) { return bars + 8u * (2 + 2 * STAGES + 2 * kAccBufs + b); };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + L::kTmemSlot);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + L::kAbort);
     float *lse_s = reinterpret_cast<float *>(base_ptr + L::kLse);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int unit = blockIdx.x / nt;
-    const int w = blockIdx.x - unit * nt;                   // heaviest tile of the unit first
-    const int stat_tile = PASS2 ? w : nt - 1 - w;
-    const int count = PASS2 ? nt - stat_tile : stat_tile + 1;
     const CUtensorMap *map_stat = PASS2 ? &map_k : &map_q;
     const CUtensorMap *map_strm = PASS2 ? &map_q : &map_k;
+    const int nts = PASS2 ? geo.ntk : geo.ntq;              // stationary tiles per unit
+    const int spu = (nts + 1) / 2;                          // item pairs per unit
 
     // a CTA of this launch has already given up: leave at once instead of timing out again
     if (threadIdx.x == 0) *abort_flag = *reinterpret_cast<volatile int *>(status);
@@ -188,7 +243,8 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (*abort_flag) return;
 
     if (threadIdx.x == 0) {
-        mbar_init(bar_stat, 1);
+        mbar_init(bar_stat_full, 1);
+        mbar_init(bar_stat_empty, 1);
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(bar_acc_full(b), 1);
@@ -208,52 +264,85 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Every role walks the same item list with the same counters: `it` counts items (stationary
+    // tiles), `tg` counts streamed tiles; ring slots and barrier phases derive from them.
+    uint32_t it = 0, tg = 0;
+    bool alive = true;
+
+    // item `sub` (0 = heavy, 1 = its complement) of pair `sidx`: stationary tile and streamed range
+    auto item_of = [&](int sidx, int sub, int &unit, int &st, int &first, int &count) -> bool {
+        unit = sidx / spu;
+        const int pi = sidx - unit * spu;
+        const int heavy = PASS2 ? pi : nts - 1 - pi, light = nts - 1 - heavy;
+        if (sub == 1 && light == heavy) return false;
+        st = sub ? light : heavy;
+        if (PASS2) { first = geo.imin(st); count = geo.ntq - first; }
+        else       { first = geo.jmax(st); count = first + 1; }
+        return true;
+    };
+    auto stream_tile = [&](int first, int t) { return PASS2 ? first + t : first - t; };
+
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            mbar_expect_tx(bar_stat, kTileBytes);
+            uint32_t armed = 0;
+            for (int sidx = blockIdx.x; alive && sidx < n_super; sidx += gridDim.x) {
+                for (int sub = 0; alive && sub < 2; ++sub) {
+                    int unit, st, first, count;
+                    if (!item_of(sidx, sub, unit, st, first, count)) break;
+                    // the stationary buffer is free once the previous item's last MMA has completed
+                    if (!mbar_wait(bar_stat_empty, (it + 1u) & 1u, abort_flag, status)) { alive = false; break; }
+                    mbar_expect_tx(bar_stat_full, kTileBytes);
 #pragma unroll
-            for (int bx = 0; bx < kBoxes; ++bx)
-                tma_load_3d(base + L::kStat + bx * kBoxBytes, map_stat, bx * 64, stat_tile * kTileRows, unit, bar_stat);
-            int armed = 0;
-            for (int t = 0; t < count; ++t) {
-                const int s = t % STAGES;
-                const uint32_t ph = (uint32_t)(t / STAGES) & 1u;
-                if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, status)) break;
-                const int tile = PASS2 ? stat_tile + t : stat_tile - t;
-                mbar_expect_tx(bar_full(s), kTileBytes);
+                    for (int bx = 0; bx < kBoxes; ++bx)
+                        tma_load_3d(base + L::kStat + bx * kBoxBytes, map_stat, bx * 64, st * kTileRows, unit, bar_stat_full);
+                    for (int t = 0; t < count; ++t, ++tg) {
+                        const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
+                        if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, status)) { alive = false; break; }
+                        mbar_expect_tx(bar_full(s), kTileBytes);
 #pragma unroll
-                for (int bx = 0; bx < kBoxes; ++bx)
-                    tma_load_3d(base + L::kStage0 + s * kTileBytes + bx * kBoxBytes, map_strm, bx * 64,
-                                tile * kTileRows, unit, bar_full(s));
-                armed = t + 1;
+                        for (int bx = 0; bx < kBoxes; ++bx)
+                            tma_load_3d(base + L::kStage0 + s * kTileBytes + bx * kBoxBytes, map_strm, bx * 64,
+                                        stream_tile(first, t) * kTileRows, unit, bar_full(s));
+                        armed = tg + 1;
+                    }
+                    ++it;
+                }
             }
             if (*abort_flag) {
                 // let copies that are still in flight land before the CTA gives its memory back
-                mbar_wait(bar_stat, 0, abort_flag, status, 200000ull);
-                for (int t = max(0, armed - STAGES); t < armed; ++t)
-                    mbar_wait(bar_full(t % STAGES), (uint32_t)(t / STAGES) & 1u, abort_flag, status, 200000ull);
+                if (it > 0) mbar_wait(bar_stat_full, (it - 1u) & 1u, abort_flag, status, 200000ull);
+                for (uint32_t t = armed > (uint32_t)STAGES ? armed - STAGES : 0; t < armed; ++t)
+                    mbar_wait(bar_full(t % STAGES), (t / STAGES) & 1u, abort_flag, status, 200000ull);
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            bool ok = mbar_wait(bar_stat, 0, abort_flag, status);
-            for (int t = 0; ok && t < count; ++t) {
-                const int s = t % STAGES, b = t % kAccBufs;
-                const uint32_t ph = (uint32_t)(t / STAGES) & 1u, bph = (uint32_t)(t / kAccBufs) & 1u;
-                if (!mbar_wait(bar_acc_empty(b), bph ^ 1u, abort_flag, status)) break;
-                if (!mbar_wait(bar_full(s), ph, abort_flag, status)) break;
-                tc_fence_after();
-                const uint32_t a0 = base + L::kStat, b0 = base + L::kStage0 + s * kTileBytes;
+            for (int sidx = blockIdx.x; alive && sidx < n_super; sidx += gridDim.x) {
+                for (int sub = 0; alive && sub < 2; ++sub) {
+                    int unit, st, first, count;
+                    if (!item_of(sidx, sub, unit, st, first, count)) break;
+                    if (!mbar_wait(bar_stat_full, it & 1u, abort_flag, status)) { alive = false; break; }
+                    for (int t = 0; t < count; ++t, ++tg) {
+                        const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
+                        const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
+                        if (!mbar_wait(bar_acc_empty(b), bph ^ 1u, abort_flag, status)) { alive = false; break; }
+                        if (!mbar_wait(bar_full(s), ph, abort_flag, status)) { alive = false; break; }
+                        tc_fence_after();
+                        const uint32_t a0 = base + L::kStat, b0 = base + L::kStage0 + s * kTileBytes;
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (uint32_t)(k / 4) * kBoxBytes + (uint32_t)(k % 4) * 32u;
-                    umma_bf16(tmem_base + (uint32_t)b * kTileRows, umma_desc(a0 + off), umma_desc(b0 + off), kIdesc,
-                              k > 0 ? 1u : 0u);
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t off = (uint32_t)(k / 4) * kBoxBytes + (uint32_t)(k % 4) * 32u;
+                            umma_bf16(tmem_base + b * kTileRows, umma_desc(a0 + off), umma_desc(b0 + off), kIdesc,
+                                      k > 0 ? 1u : 0u);
+                        }
+                        umma_commit(bar_empty(s));       // stage reusable once these MMAs have read it
+                        umma_commit(bar_acc_full(b));    // accumulator ready for the softmax warps
+                    }
+                    if (alive) umma_commit(bar_stat_empty);   // stationary tile no longer read
+                    ++it;
                 }
-                umma_commit(bar_empty(s));       // stage reusable once these MMAs have read it
-                umma_commit(bar_acc_full(b));    // accumulator ready for the softmax warps
             }
         }
     } else {
@@ -261,76 +350,103 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int q4 = warp & 3;                              // TMEM lane quarter this warp may read
         const int r = q4 * 32 + lane;                         // row of the stationary tile = TMEM lane
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
-        const size_t lse_row = (size_t)unit * nt * kTileRows;
-        float mrun = -INFINITY, Z = 0.f;                      // pass 1 running max / sum (log2 domain)
-        float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f; // pass 2 column sum
-        bool ok = true;
-        for (int t = 0; t < count; ++t) {
-            const int b = t % kAccBufs;
-            const uint32_t bph = (uint32_t)(t / kAccBufs) & 1u;
-            if (PASS2) {
-                const int tile = stat_tile + t;
-                // every softmax thread stages one entry of the tile's lse, then all wait (bounded) for
-                // the 128 entries; the buffer is reused two tiles later, after the next tile's rendezvous
-                lse_s[b * kTileRows + r] = lse2[lse_row + (size_t)tile * kTileRows + r];
-                mbar_arrive(bar_lse(b));
-                if (!mbar_wait(bar_lse(b), bph, abort_flag, status)) { ok = false; break; }
-            }
-            if (!mbar_wait(bar_acc_full(b), bph, abort_flag, status)) { ok = false; break; }
-            tc_fence_after();
-            const bool diag = (t == 0);
-#pragma unroll 1
-            for (int ch = 0; ch < kTileRows / 32; ++ch) {
-                float v[32];
-                tmem_ld32(lane_addr + (uint32_t)(b * kTileRows + ch * 32), v);
-                if (!PASS2) {
-                    if (diag) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) if (ch * 32 + i > r) v[i] = -INFINITY;   // key n <= query m
+        const int Tk = geo.Tk();
+        for (int sidx = blockIdx.x; alive && sidx < n_super; sidx += gridDim.x) {
+            for (int sub = 0; alive && sub < 2; ++sub) {
+                int unit, st, first, count;
+                if (!item_of(sidx, sub, unit, st, first, count)) break;
+                const size_t lse_row = (size_t)unit * geo.ntq * kTileRows;
+                float mrun = -INFINITY, Z = 0.f;                      // pass 1 running max / sum (log2 domain)
+                float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f; // pass 2 column sum
+                for (int t = 0; t < count; ++t, ++tg) {
+                    const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
+                    const int tile = stream_tile(first, t);
+                    // off = 128*(query tile - key tile) + P: element (row, col) is visible iff
+                    //   pass 1 (row = query, col = key):  col <= row + off
+                    //   pass 2 (row = key,  col = query): col >= row - off
+                    const int off = (PASS2 ? tile - st : st - tile) * kTileRows + geo.P;
+                    const bool masked = off < kTileRows - 1;
+                    if (PASS2) {
+                        // every softmax thread stages one entry of the tile's lse, then all wait (bounded)
+                        // for the 128 entries; the buffer is reused two tiles later, after the next
+                        // tile's rendezvous
+                        lse_s[b * kTileRows + r] = lse2[lse_row + (size_t)tile * kTileRows + r];
+                        mbar_arrive(bar_lse(b));
+                        if (!mbar_wait(bar_lse(b), bph, abort_flag, status)) { alive = false; break; }
                     }
-                    float cm = v[0];
+                    if (!mbar_wait(bar_acc_full(b), bph, abort_flag, status)) { alive = false; break; }
+                    tc_fence_after();
+
+                    auto chunk = [&](uint32_t (&raw)[32], int ch) {
+                        float v[32];
 #pragma unroll
-                    for (int i = 1; i < 32; ++i) cm = fmaxf(cm, v[i]);
-                    const float mnew = fmaxf(mrun, cm * c);
-                    if (mnew != -INFINITY) {
-                        float part[4] = {0.f, 0.f, 0.f, 0.f};
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]);
+                        if (!PASS2) {
+                            if (masked) {
+                                const int lim = r + off - ch * 32;            // columns i <= lim are visible
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) part[i & 3] += fast_exp2(fmaf(v[i], c, -mnew));
-                        Z = Z * fast_exp2(mrun - mnew) + ((part[0] + part[1]) + (part[2] + part[3]));
-                        mrun = mnew;
-                    }
-                } else {
-                    const float4 *ls = reinterpret_cast<const float4 *>(lse_s + b * kTileRows + ch * 32);
+                                for (int i = 0; i < 32; ++i) if (i > lim) v[i] = -INFINITY;
+                            }
+                            float cm = v[0];
 #pragma unroll
-                    for (int i4 = 0; i4 < 8; ++i4) {
-                        const float4 l4 = ls[i4];
-                        float p0 = fast_exp2(fmaf(v[i4 * 4 + 0], c, -l4.x));
-                        float p1 = fast_exp2(fmaf(v[i4 * 4 + 1], c, -l4.y));
-                        float p2 = fast_exp2(fmaf(v[i4 * 4 + 2], c, -l4.z));
-                        float p3 = fast_exp2(fmaf(v[i4 * 4 + 3], c, -l4.w));
-                        if (diag) {                                                       // query m >= key n
-                            const int c0 = ch * 32 + i4 * 4;
-                            if (c0 + 0 < r) p0 = 0.f;
-                            if (c0 + 1 < r) p1 = 0.f;
-                            if (c0 + 2 < r) p2 = 0.f;
-                            if (c0 + 3 < r) p3 = 0.f;
+                            for (int i = 1; i < 32; ++i) cm = fmaxf(cm, v[i]);
+                            const float mnew = fmaxf(mrun, cm * c);
+                            if (mnew != -INFINITY) {
+                                float part[4] = {0.f, 0.f, 0.f, 0.f};
+                                sum_exp2<0>(v, c, mnew, part);
+                                Z = Z * fast_exp2(mrun - mnew) + ((part[0] + part[1]) + (part[2] + part[3]));
+                                mrun = mnew;
+                            }
+                        } else {
+                            const float4 *ls = reinterpret_cast<const float4 *>(lse_s + b * kTileRows + ch * 32);
+                            const int lim = r - off - ch * 32;                // columns i >= lim are visible
+#pragma unroll
+                            for (int i4 = 0; i4 < 8; ++i4) {
+                                const float4 l4 = ls[i4];
+                                float p0 = exp2_mixed<0>(fmaf(v[i4 * 4 + 0], c, -l4.x));
+                                float p1 = exp2_mixed<1>(fmaf(v[i4 * 4 + 1], c, -l4.y));
+                                float p2 = exp2_mixed<2>(fmaf(v[i4 * 4 + 2], c, -l4.z));
+                                float p3 = exp2_mixed<3>(fmaf(v[i4 * 4 + 3], c, -l4.w));
+                                if (masked) {
+                                    if (i4 * 4 + 0 < lim) p0 = 0.f;
+                                    if (i4 * 4 + 1 < lim) p1 = 0.f;
+                                    if (i4 * 4 + 2 < lim) p2 = 0.f;
+                                    if (i4 * 4 + 3 < lim) p3 = 0.f;
+                                }
+                                acc0 += p0; acc1 += p1; acc2 += p2; acc3 += p3;
+                            }
                         }
-                        acc0 += p0; acc1 += p1; acc2 += p2; acc3 += p3;
-                    }
+                    };
+
+                    // the load of the next 32 columns is in flight while the current ones are processed
+                    const uint32_t col0 = lane_addr + b * kTileRows;
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32_async(col0, ra);
+                    tmem_ld_wait(ra);
+                    tmem_ld32_async(col0 + 32, rb);
+                    chunk(ra, 0);
+                    tmem_ld_wait(rb);
+                    tmem_ld32_async(col0 + 64, ra);
+                    chunk(rb, 1);
+                    tmem_ld_wait(ra);
+                    tmem_ld32_async(col0 + 96, rb);
+                    chunk(ra, 2);
+                    tmem_ld_wait(rb);
+                    tc_fence_before();                   // all TMEM reads of this tile are done:
+                    __syncwarp();                        // hand the accumulator back before the last chunk's math
+                    if (lane == 0) mbar_arrive(bar_acc_empty(b));
+                    chunk(rb, 3);
                 }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty(b));
-        }
-        if (ok) {
-            const int row = stat_tile * kTileRows + r;
-            if (!PASS2) {
-                const float l2 = (row < T) ? mrun + __log2f(Z) : INFINITY;
-                lse2[lse_row + row] = l2;
-                if (lse_out && row < T) lse_out[(size_t)unit * T + row] = l2 * kLn2;
-            } else if (row < T) {
-                scores[(size_t)unit * T + row] = (acc0 + acc1) + (acc2 + acc3);
+                if (!alive) break;
+                const int row = st * kTileRows + r;
+                if (!PASS2) {
+                    const float l2 = (row < geo.Tq) ? mrun + __log2f(Z) : INFINITY;
+                    lse2[lse_row + row] = l2;
+                    if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
+                } else if (row < Tk) {
+                    scores[(size_t)unit * Tk + row] = (acc0 + acc1) + (acc2 + acc3);
+                }
+                ++it;
             }
         }
     }
@@ -384,19 +500,30 @@ __global__ void lse_import_kernel(const float *__restrict__ lse_nat, float *__re
     lse2[(size_t)unit * Tpad + m] = (m < T) ? lse_nat[(size_t)unit * T + m] * kLog2e : INFINITY;
 }
 
+int sm_count()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 148;
+    return n;
+}
+
 template <int D, int STAGES>
-cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int units, int T, int nt, float c, float *lse2,
-                          float *lse_out, float *scores, int *status, bool first_pass, cudaStream_t stream)
+cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int units, const Geometry &geo, float c,
+                          float *lse2, float *lse_out, float *scores, int *status, bool first_pass, cudaStream_t stream)
 {
     constexpr int smem = Smem<D, STAGES>::kDynBytes;
     cudaError_t e = cudaFuncSetAttribute(importance_kernel<D, STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(importance_kernel<D, STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)units * (unsigned)nt;
+    const long long resident = 2LL * sm_count();              // two persistent CTAs per SM
+    const long long super1 = (long long)units * ((geo.ntq + 1) / 2), super2 = (long long)units * ((geo.ntk + 1) / 2);
     if (first_pass)
-        importance_kernel<D, STAGES, false><<<grid, kThreads, smem, stream>>>(mq, mk, T, nt, c, lse2, lse_out, scores, status);
-    importance_kernel<D, STAGES, true><<<grid, kThreads, smem, stream>>>(mq, mk, T, nt, c, lse2, lse_out, scores, status);
+        importance_kernel<D, STAGES, false><<<(unsigned)(super1 < resident ? super1 : resident), kThreads, smem, stream>>>(
+            mq, mk, geo, (int)super1, c, lse2, lse_out, scores, status);
+    importance_kernel<D, STAGES, true><<<(unsigned)(super2 < resident ? super2 : resident), kThreads, smem, stream>>>(
+        mq, mk, geo, (int)super2, c, lse2, lse_out, scores, status);
     return cudaGetLastError();
 }
 
@@ -410,27 +537,32 @@ size_t importance_workspace_bytes(int N, int H, int T, int D)
 }
 
 // lse_in == nullptr: both passes. Otherwise the caller's normaliser replaces pass 1.
+// Q: [units, Tq, D]; K: [units, P + Tq, D]; scores: [units, P + Tq]; lse_out / lse_in: [units, Tq].
 cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out, const float *lse_in,
-                              int N, int H, int T, int D, float scale, void *ws, cudaStream_t stream)
+                              int N, int H, int Tq, int P, int D, float scale, void *ws, cudaStream_t stream)
 {
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return e;
     int *status = static_cast<int *>(ws);
     float *lse2 = reinterpret_cast<float *>(static_cast<char *>(ws) + kStatusBytes);
     const int units = N * H;
-    const int nt = (T + kTileRows - 1) / kTileRows;
-    if ((long long)units * nt > 0x7FFFFFFFLL || units > 65535 * 1024) return cudaErrorInvalidConfiguration;
+    Geometry geo;
+    geo.Tq = Tq;
+    geo.P = P;
+    geo.ntq = (Tq + kTileRows - 1) / kTileRows;
+    geo.ntk = (Tq + P + kTileRows - 1) / kTileRows;
+    if ((long long)units * geo.ntk > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     CUtensorMap mq, mk;
-    if (!make_map(&mq, Q, units, T, D) || !make_map(&mk, K, units, T, D)) return cudaErrorInvalidValue;
+    if (!make_map(&mq, Q, units, Tq, D) || !make_map(&mk, K, units, Tq + P, D)) return cudaErrorInvalidValue;
     if (lse_in) {
         if (units > 65535) return cudaErrorInvalidConfiguration;
-        dim3 g((nt * kTileRows + 255) / 256, units);
-        lse_import_kernel<<<g, 256, 0, stream>>>(lse_in, lse2, T, nt * kTileRows);
+        dim3 g((geo.ntq * kTileRows + 255) / 256, units);
+        lse_import_kernel<<<g, 256, 0, stream>>>(lse_in, lse2, Tq, geo.ntq * kTileRows);
     }
     const float c = scale * kLog2e;
     if (D == 128)
-        return launch_passes<128, 2>(mq, mk, units, T, nt, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
-    return launch_passes<64, 4>(mq, mk, units, T, nt, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
+        return launch_passes<128, 2>(mq, mk, units, geo, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
+    return launch_passes<64, 4>(mq, mk, units, geo, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
 }
 
 }  // namespace ec

@@ -344,3 +344,24 @@ def test_group_mean_and_gather_reduce_to_numpy():
     X = wl.bf16_bits_to_f64(Xb)
     for u in range(2):
         np.testing.assert_array_equal(got[u], X[u, a[u]])
+
+
+def test_importance_prefix_matches_library_softmax_and_reduces_to_plain():
+    rng = np.random.default_rng(41)
+    for Tq, P, D in [(1, 0, 4), (5, 3, 4), (17, 40, 8), (30, 1, 8)]:
+        qb, kb = _rand_bits(rng, (2, Tq, D)), _rand_bits(rng, (2, P + Tq, D))
+        scores, lse = orc.importance_prefix(qb, kb, 0.4)
+        q = torch.from_numpy(wl.bf16_bits_to_f64(qb))
+        k = torch.from_numpy(wl.bf16_bits_to_f64(kb))
+        logits = 0.4 * q @ k.transpose(-1, -2)                           # [2, Tq, P+Tq]
+        m_idx = torch.arange(Tq)[:, None]
+        n_idx = torch.arange(P + Tq)[None, :]
+        logits = logits.masked_fill(n_idx > m_idx + P, float("-inf"))     # query m sees keys n <= m + P
+        A = torch.softmax(logits, dim=-1)
+        np.testing.assert_allclose(scores, A.sum(dim=-2).numpy(), rtol=1e-12)
+        np.testing.assert_allclose(lse, torch.logsumexp(logits, dim=-1).numpy(), rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(scores.sum(-1), Tq, rtol=1e-12)       # one unit of mass per query
+        if P == 0:
+            s0, l0 = orc.importance(qb, kb, 0.4)
+            np.testing.assert_array_equal(scores, s0)
+            np.testing.assert_array_equal(lse, l0)

@@ -496,3 +496,24 @@ def test_decode_steps_overlapped_loop_with_many_units():
                                     policy=orc.POLICY_FIXED, budget=C, offset=d)
             err = np.abs(b[s, n, h] - want[0])
             assert (err <= 2e-2 + 2.0 ** -8 * np.abs(want[0])).all(), (n, h, s)
+
+
+# ---------------------------------------------------------------- importance over cache + new instruction
+
+@pytest.mark.parametrize("N,H,Tq,P,D", [(1, 2, 1, 5, 64), (1, 2, 130, 1, 128), (2, 2, 200, 127, 128), (1, 3, 129, 128, 64),
+                                        (1, 2, 300, 333, 128), (1, 1, 64, 700, 128), (1, 2, 640, 320, 128)])
+def test_importance_prefix_matches_oracle(N, H, Tq, P, D):
+    rng = np.random.default_rng(Tq + 3 * P)
+    Qb, Kb = rand_bits(rng, (N, H, Tq, D)), rand_bits(rng, (N, H, P + Tq, D))
+    scale = 1.0 / math.sqrt(D)
+    want, want_lse = orc.importance_prefix(Qb, Kb, scale)
+    scores = Guarded((N, H, P + Tq), torch.float32, fill=float("nan"))
+    lse = Guarded((N, H, Tq), torch.float32, fill=float("nan"))
+    ws = scratch(ec.ec_importance_workspace(N, H, Tq, D))
+    ec.ec_importance_prefix(dev_bf16(Qb), dev_bf16(Kb), scores.t, lse.t, scale, ws)
+    assert ec.ec_device_status(ws) == ec.EC_OK
+    scores.check("scores")
+    lse.check("lse")
+    assert_rel_close(scores.t, want, SCORE_RTOL, what="scores with prefix")
+    assert_rel_close(lse.t, want_lse, 1e-3, atol=1e-3, what="lse with prefix")
+    np.testing.assert_allclose(host_f64(scores.t).sum(-1), Tq, rtol=1e-3)
