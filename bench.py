@@ -396,6 +396,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llava7b_b1", choices=list(wl.WORKLOADS))
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode length")
+    ap.add_argument("--problems", type=int, default=None,
+                    help="run only the first K problems (batch x layer pairs) of the workload: for profiling captures")
     ap.add_argument("--oracle-decode-steps", type=int, default=0)
     ap.add_argument("--oracle-problems", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -403,6 +405,8 @@ def main():
     w = wl.WORKLOADS[args.workload]
     if args.decode_steps:
         w = w.shrunk(decode_steps=args.decode_steps)
+    if args.problems:
+        w = w.shrunk(batch=1, layers=min(args.problems, w.N))      # problem n keeps its own draws
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -139,10 +139,12 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32])
 }
 
 // 2^x on the FMA pipe (Cody-Waite split + degree-4 polynomial, relative error < 6e-6) for
-// x <= ~0. One element in EC_IMP_POLY_EVERY goes this way, to take some load off the
+// x <= ~0. With EC_IMP_POLY_EVERY = n > 0, one element in n goes this way to take load off the
 // special-function unit (one ex2 per score element is the busiest pipe of these kernels).
+// Off by default: measured on B200 it does not pay (n = 4: -1..+1%, n = 3: -5%), because with
+// two CTAs per SM the softmax warps wait on TMEM loads and barriers more than on the ex2 pipe.
 #ifndef EC_IMP_POLY_EVERY
-#define EC_IMP_POLY_EVERY 4          // 0 = never
+#define EC_IMP_POLY_EVERY 0          // 0 = never
 #endif
 __device__ __forceinline__ float poly_exp2(float x)
 {
