@@ -122,6 +122,16 @@ int ec_importance_from_lse(const void *Q_dev, const void *K_dev, const float *ls
  */
 int ec_device_status(void *ws_dev, void *stream);
 
+/*
+ * Self-test of the failure path (no counterpart in the paper). The importance kernels wait
+ * on hardware barriers with a time limit so that a lost signal can never hang the GPU. This
+ * call enqueues a one-CTA kernel that waits, with that same routine, on a barrier nothing
+ * completes; after `limit_us` microseconds (1 .. 1 000 000) the wait gives up, sets the status
+ * word of `ws_dev` (any 256-byte-aligned device buffer of >= 256 bytes) and the kernel ends
+ * normally. ec_device_status(ws_dev) then reports EC_ERR_TIMEOUT; the context stays usable.
+ */
+int ec_selftest_wait_timeout(void *ws_dev, unsigned limit_us, void *stream);
+
 /* ---------------------------------------------------------------- select + merge ---- */
 
 typedef enum {

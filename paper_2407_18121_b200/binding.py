@@ -22,7 +22,7 @@ EC_LAYER_SHARED = 1
 
 EXPORTS = (
     "ec_status_string", "ec_keep_count",
-    "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_from_lse", "ec_device_status",
+    "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_from_lse", "ec_device_status", "ec_selftest_wait_timeout",
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
     "ec_cache_init", "ec_cache_init_ratio", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc",
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
     L.ec_importance_from_lse.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
     L.ec_device_status.restype = i
     L.ec_device_status.argtypes = [vp, vp]
+    L.ec_selftest_wait_timeout.restype = i
+    L.ec_selftest_wait_timeout.argtypes = [vp, C.c_uint, vp]
     L.ec_select_merge_workspace.restype = sz
     L.ec_select_merge_workspace.argtypes = [i, i, i, i, i, i]
     L.ec_select_merge.restype = i
@@ -161,6 +163,11 @@ def ec_importance_from_lse(Q: torch.Tensor, K: torch.Tensor, lse: torch.Tensor, 
 
 def ec_device_status(ws: torch.Tensor) -> int:
     return int(lib().ec_device_status(_ptr(ws), _stream()))
+
+
+def ec_selftest_wait_timeout(ws: torch.Tensor, limit_us: int) -> None:
+    """Enqueue the bounded-wait self-test: afterwards ec_device_status(ws) reports EC_ERR_TIMEOUT."""
+    _check(lib().ec_selftest_wait_timeout(_ptr(ws), int(limit_us), _stream()), "ec_selftest_wait_timeout")
 
 
 def ec_select_merge_workspace(N: int, H: int, T: int, D: int, n_keep: int, population: int) -> int:

@@ -103,6 +103,14 @@ int ec_importance_from_lse(const void *Q, const void *K, const float *lse, float
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 
+int ec_selftest_wait_timeout(void *ws, unsigned limit_us, void *stream)
+{
+    if (!ws) return EC_ERR_NULL;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    if (limit_us < 1 || limit_us > 1000000u) return EC_ERR_ARG;
+    return ec::launch_wait_selftest(ws, limit_us, (cudaStream_t)stream) == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
 int ec_device_status(void *ws, void *stream)
 {
     if (!ws) return EC_ERR_NULL;

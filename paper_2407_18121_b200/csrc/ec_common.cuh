@@ -59,6 +59,7 @@ __device__ __forceinline__ float fast_exp2(float x)
 cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out, const float *lse_in,
                               int N, int H, int Tq, int P, int D, float scale, void *ws, cudaStream_t stream);
 size_t importance_workspace_bytes(int N, int H, int T, int D);
+cudaError_t launch_wait_selftest(void *ws, unsigned limit_us, cudaStream_t stream);
 
 cudaError_t launch_select(const float *scores, int units, int T, int n_keep, int share, int protect_ends,
                           int32_t *anchor_pos, int32_t *bucket_len, float *mean_ws, cudaStream_t stream);

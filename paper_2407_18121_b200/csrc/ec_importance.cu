@@ -502,6 +502,21 @@ __global__ void lse_import_kernel(const float *__restrict__ lse_nat, float *__re
     lse2[(size_t)unit * Tpad + m] = (m < T) ? lse_nat[(size_t)unit * T + m] * kLog2e : INFINITY;
 }
 
+// One CTA waits, with the same bounded wait the importance kernels use, on a barrier that
+// nothing ever completes: the wait has to expire, flag the status word and let the kernel end.
+__global__ void wait_selftest_kernel(int *status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, &abort_flag, status, limit_ns);
+}
+
 int sm_count()
 {
     int dev = 0, n = 0;
@@ -530,6 +545,14 @@ cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int unit
 }
 
 }  // namespace
+
+cudaError_t launch_wait_selftest(void *ws, unsigned limit_us, cudaStream_t stream)
+{
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, stream);
+    if (e != cudaSuccess) return e;
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(static_cast<int *>(ws), (unsigned long long)limit_us * 1000ull);
+    return cudaGetLastError();
+}
 
 size_t importance_workspace_bytes(int N, int H, int T, int D)
 {

@@ -61,6 +61,38 @@ class ElasticCacheSession:
         """Generation calls for q, k_new, v_new, out of shape [steps, N, H, D]."""
         return ec.ec_decode_steps(q, k_new, v_new, self.cache, self.scale, out, self.ws_dec, want_slots)
 
+    # ---- a new instruction on top of the current cache ---------------------------------
+    def logical_slots(self):
+        """Physical slots of the cache rows in queue order (oldest first), fixed-budget policy:
+        the rows before the ring never move; the ring holds the `offset` newest rows, oldest at
+        `ring_head`."""
+        c = self.cache
+        if c.policy != 0:
+            raise ValueError("queue order is only tracked for the fixed-budget policy")
+        if c.len < c.budget:
+            return list(range(c.len))
+        base = c.budget - c.offset
+        return list(range(base)) + [base + (c.ring_head + i) % c.offset for i in range(c.offset)]
+
+    def recompress(self, Q_new: torch.Tensor, K_new: torch.Tensor, V_new: torch.Tensor, keep_ratio: float):
+        """Encode a new instruction of Tq tokens on top of the cache: importance of the cached rows and
+        the new rows under the new tokens' queries, then selection and merge over the concatenation.
+        Returns a new session holding the compacted result (this one is left untouched)."""
+        N, H, Tq, D = Q_new.shape
+        idx = torch.tensor(self.logical_slots(), dtype=torch.long, device=self.device)
+        K_all = torch.cat([self.Kc.index_select(2, idx), K_new], dim=2).contiguous()
+        V_all = torch.cat([self.Vc.index_select(2, idx), V_new], dim=2).contiguous()
+        P = idx.numel()
+        nxt = ElasticCacheSession(N, H, P + Tq, D, keep_ratio, self.offset, self.scale, self.population,
+                                  self.protect_ends, device=self.device)
+        ws = torch.empty(ec.ec_importance_workspace(N, H, Tq, D), dtype=torch.uint8, device=self.device)
+        ec.ec_importance_prefix(Q_new, K_all, nxt.scores, None, self.scale, ws)
+        ec.ec_select_merge(K_all, V_all, nxt.scores, nxt.n_keep, nxt.population, nxt.protect_ends,
+                           nxt.Kc, nxt.Vc, nxt.anchor_pos, None, nxt.ws_sel)
+        nxt.cache = ec.ec_cache_init(nxt.Kc, nxt.Vc, nxt.n_keep, max(nxt.n_keep, 2),
+                                     min(nxt.offset, max(nxt.n_keep, 2) - 1))
+        return nxt
+
     # ---- host-resident inputs --------------------------------------------------------
     def _prompt_staging(self):
         if self._stage is None:

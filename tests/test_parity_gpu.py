@@ -517,3 +517,80 @@ def test_importance_prefix_matches_oracle(N, H, Tq, P, D):
     assert_rel_close(scores.t, want, SCORE_RTOL, what="scores with prefix")
     assert_rel_close(lse.t, want_lse, 1e-3, atol=1e-3, what="lse with prefix")
     np.testing.assert_allclose(host_f64(scores.t).sum(-1), Tq, rtol=1e-3)
+
+
+# ---------------------------------------------------------------- failure path of the bounded waits
+
+def test_bounded_wait_expires_reports_and_leaves_the_context_usable():
+    """A barrier that nothing completes: the wait gives up after its limit, the status word says so,
+    and the next real call on the same workspace runs normally (no hang, no fault)."""
+    rng = np.random.default_rng(2)
+    N, H, T, D = 1, 2, 200, 128
+    ws = scratch(ec.ec_importance_workspace(N, H, T, D))
+    ec.ec_selftest_wait_timeout(ws, 2000)                       # 2 ms
+    assert ec.ec_device_status(ws) == 7                         # EC_ERR_TIMEOUT
+    assert "timed out" in ec.status_string(7)
+    Qb, Kb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+    want, _ = orc.importance(Qb, Kb, 0.1)
+    scores = torch.empty((N, H, T), dtype=torch.float32, device="cuda")
+    ec.ec_importance(dev_bf16(Qb), dev_bf16(Kb), scores, None, 0.1, ws)
+    assert ec.ec_device_status(ws) == ec.EC_OK                  # the status word is reset by every call
+    assert_rel_close(scores, want, SCORE_RTOL, what="scores after a timed-out self-test")
+
+
+# ---------------------------------------------------------------- a second instruction on top of the cache
+
+def test_second_instruction_on_top_of_a_decoded_cache():
+    """Prompt -> compact -> decode -> a new instruction arrives -> compact [cache ; new rows] -> decode.
+    The oracle runs its own chain; the GPU's second stage starts from the oracle's queue (rows placed
+    in ring order, as a decoded cache holds them), so both sides see identical inputs."""
+    from paper_2407_18121_b200.session import ElasticCacheSession
+    rng = np.random.default_rng(99)
+    N, H, D, C, d, S1, Tq, S2, scale, ratio = 1, 4, 128, 64, 16, 21, 150, 6, 0.09, 0.5
+    # oracle stage 1: a compacted cache of C rows, S1 decode steps
+    K0b, V0b = rand_bits(rng, (N, H, C, D)), rand_bits(rng, (N, H, C, D))
+    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=C + 1)
+    for s in range(S1):
+        qb, kb, vb = (rand_bits(rng, (N, H, D)) for _ in range(3))
+        queue.step(qb, kb, vb, scale, policy=orc.POLICY_FIXED, budget=C, offset=d)
+    Kq = orc.round_bf16(queue.K[:, :C].reshape(N, H, C, D))          # queue order, exact (rows are bf16 values)
+    Vq = orc.round_bf16(queue.V[:, :C].reshape(N, H, C, D))
+
+    # the same cache as the GPU holds it after S1 evictions: ring rotated by S1 mod d
+    sess = ElasticCacheSession(N, H, 2 * C, D, 0.5, d, scale)          # n_keep = C
+    assert sess.n_keep == C
+    head = S1 % d
+    phys = list(range(C - d)) + [C - d + (i - head) % d for i in range(d)]   # queue position -> slot offset
+    Kp, Vp = np.empty_like(Kq), np.empty_like(Vq)
+    for pos in range(C):
+        slot = pos if pos < C - d else C - d + (head + (pos - (C - d))) % d
+        Kp[:, :, slot], Vp[:, :, slot] = Kq[:, :, pos], Vq[:, :, pos]
+    sess.Kc[:, :, :C] = dev_bf16(Kp)
+    sess.Vc[:, :, :C] = dev_bf16(Vp)
+    sess.cache = ec.ec_cache_init(sess.Kc, sess.Vc, C, C, d)
+    sess.cache.ring_head = head
+    order = sess.logical_slots()
+    np.testing.assert_array_equal(host_bits(sess.Kc[:, :, order]), Kq)    # queue order recovered
+
+    # the new instruction
+    Qn, Kn, Vn = (rand_bits(rng, (N, H, Tq, D)) for _ in range(3))
+    K_all, V_all = np.concatenate([Kq, Kn], 2), np.concatenate([Vq, Vn], 2)
+    o_scores, _ = orc.importance_prefix(Qn, K_all, scale)
+    C2 = orc.keep_count(C + Tq, ratio)
+    o_anch = orc.select(o_scores, C2, True)
+    nxt = sess.recompress(dev_bf16(Qn), dev_bf16(Kn), dev_bf16(Vn), ratio)
+    assert nxt.n_keep == C2
+    assert_rel_close(nxt.scores, o_scores, SCORE_RTOL, what="scores over cache + new instruction")
+    check_anchor_sets(nxt.anchor_pos, o_anch, o_scores, C2, True)
+    lo, hi = orc.buckets(anchors_to_merge_on(nxt.anchor_pos, o_anch), C + Tq)
+    o_K, o_V = orc.merge(K_all, lo, hi), orc.merge(V_all, lo, hi)
+    assert_bf16_close(nxt.Kc, o_K, "re-merged K")
+    assert_bf16_close(nxt.Vc, o_V, "re-merged V")
+
+    queue2 = orc.DecodeQueue(orc.widen_bf16(orc.round_bf16(o_K)), orc.widen_bf16(orc.round_bf16(o_V)), cap=C2 + 1)
+    out = torch.empty((N, H, D), dtype=torch.bfloat16, device="cuda")
+    for s in range(S2):
+        qb, kb, vb = (rand_bits(rng, (N, H, D)) for _ in range(3))
+        want, _, _ = queue2.step(qb, kb, vb, scale, policy=orc.POLICY_FIXED, budget=C2, offset=d)
+        ec.ec_decode_step(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), nxt.cache, scale, out, nxt.ws_dec)
+        assert_bf16_close(out, want, f"decode after the second instruction, step {s}")
