@@ -272,6 +272,41 @@ int ec_decode_steps(const void *q_dev, const void *k_new_dev, const void *v_new_
                     ec_cache *c, float scale, void *out_dev, int *evicted_slots_host,
                     void *ws_dev, size_t ws_bytes, void *stream);
 
+/* ---------------------------------------------------------------- host-resident tensors */
+
+/*
+ * The prompt call for tensors that start in host memory (Algorithm 1's prompt branch end to
+ * end): copies Q, K, V to the caller's device staging buffers, then ec_importance and
+ * ec_select_merge, then (optionally) copies the index map back. Everything is enqueued on
+ * `stream`; pinned host memory makes the copies asynchronous.
+ *   Q_host, K_host, V_host   host bf16 [N, H, T, D]                        (in)
+ *   Q_dev, K_dev, V_dev      device staging of the same size                (scratch)
+ *   anchor_pos_host          host int32 [N, H, n_keep]; may be NULL         (out, optional)
+ *   ws_imp / ws_sel          workspaces of ec_importance / ec_select_merge
+ * Other arguments as in those two calls.
+ */
+int ec_compress_host(const void *Q_host, const void *K_host, const void *V_host,
+                     void *Q_dev, void *K_dev, void *V_dev, float *scores_dev,
+                     int N, int H, int T, int D, float scale, int n_keep, int population, int protect_ends,
+                     void *Kc_dev, void *Vc_dev, int cap, int32_t *anchor_pos_dev, int32_t *anchor_pos_host,
+                     void *ws_imp_dev, size_t ws_imp_bytes, void *ws_sel_dev, size_t ws_sel_bytes, void *stream);
+
+/*
+ * ec_decode_steps for inputs and outputs in host memory. The steps are cut into chunks of
+ * `chunk` steps (at most 31 chunks per call): the upload of later chunks (on upload_stream)
+ * and the download of finished chunks (on download_stream) overlap the decoding of the
+ * current chunk on `stream`. `stream` waits for the last download before the call's work
+ * counts as complete on it.
+ *   q_host, k_host, v_host, out_host   host bf16 [steps, N, H, D] (pinned for overlap)
+ *   q_dev, k_dev, v_dev, out_dev       device staging of the same size
+ *   upload_stream, download_stream     two further cudaStream_t, distinct from `stream`
+ * The events the call creates are destroyed before it returns.
+ */
+int ec_decode_steps_host(const void *q_host, const void *k_host, const void *v_host, void *out_host,
+                         void *q_dev, void *k_dev, void *v_dev, void *out_dev, int steps, int chunk,
+                         ec_cache *c, float scale, void *ws_dev, size_t ws_bytes,
+                         void *stream, void *upload_stream, void *download_stream);
+
 /* ---------------------------------------------------------------- no-allocation decode */
 
 /*

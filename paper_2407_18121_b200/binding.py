@@ -25,7 +25,7 @@ EXPORTS = (
     "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_from_lse", "ec_device_status", "ec_selftest_wait_timeout",
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
     "ec_cache_init", "ec_cache_init_ratio", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
-    "ec_decode_noalloc_capacity", "ec_decode_step_noalloc",
+    "ec_decode_noalloc_capacity", "ec_decode_step_noalloc", "ec_compress_host", "ec_decode_steps_host",
 )
 
 
@@ -93,6 +93,10 @@ def lib() -> C.CDLL:
     L.ec_decode_step.argtypes = [vp, vp, vp, C.POINTER(ec_cache), f, vp, C.POINTER(i), C.POINTER(i), vp, sz, vp]
     L.ec_decode_steps.restype = i
     L.ec_decode_steps.argtypes = [vp, vp, vp, i, C.POINTER(ec_cache), f, vp, C.POINTER(i), vp, sz, vp]
+    L.ec_compress_host.restype = i
+    L.ec_compress_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, i, i, vp, vp, i, vp, vp, vp, sz, vp, sz, vp]
+    L.ec_decode_steps_host.restype = i
+    L.ec_decode_steps_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, C.POINTER(ec_cache), f, vp, sz, vp, vp, vp]
     L.ec_decode_noalloc_capacity.restype = sz
     L.ec_decode_noalloc_capacity.argtypes = []
     L.ec_decode_step_noalloc.restype = i
@@ -273,3 +277,34 @@ def ec_decode_step_noalloc(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Te
                                       C.byref(ev), C.byref(sl), _stream())
     _check(st, "ec_decode_step_noalloc")
     return ev.value, sl.value
+
+
+def _host_ptr(t: torch.Tensor) -> int:
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError("a contiguous host tensor is required")
+    return t.data_ptr()
+
+
+def ec_compress_host(Q_host, K_host, V_host, Q, K, V, scores, scale: float, n_keep: int, population: int,
+                     protect_ends: bool, Kc, Vc, anchor_pos, anchor_pos_host, ws_imp, ws_sel) -> None:
+    """Prompt call from host tensors (bf16 [N,H,T,D], pinned for asynchronous copies): upload into the
+    device staging tensors Q, K, V, importance, selection + merge, optional download of the index map."""
+    N, H, T, D = Q.shape
+    st = lib().ec_compress_host(_host_ptr(Q_host), _host_ptr(K_host), _host_ptr(V_host), _ptr(Q), _ptr(K), _ptr(V),
+                                _ptr(scores), N, H, T, D, float(scale), int(n_keep), int(population),
+                                int(bool(protect_ends)), _ptr(Kc), _ptr(Vc), Kc.shape[2], _ptr(anchor_pos),
+                                None if anchor_pos_host is None else _host_ptr(anchor_pos_host),
+                                _ptr(ws_imp), ws_imp.numel(), _ptr(ws_sel), ws_sel.numel(), _stream())
+    _check(st, "ec_compress_host")
+
+
+def ec_decode_steps_host(q_host, k_host, v_host, out_host, q, k, v, out, cache: ec_cache, scale: float, ws,
+                         upload_stream: torch.cuda.Stream, download_stream: torch.cuda.Stream, chunk: int = 64) -> None:
+    """Decode loop from host tensors [steps,N,H,D]: chunked uploads and downloads on two side streams overlap
+    the decoding on the current stream; q, k, v, out are device staging tensors of the same shape."""
+    steps = q_host.shape[0]
+    st = lib().ec_decode_steps_host(_host_ptr(q_host), _host_ptr(k_host), _host_ptr(v_host), _host_ptr(out_host),
+                                    _ptr(q), _ptr(k), _ptr(v), _ptr(out), steps, int(chunk), C.byref(cache),
+                                    float(scale), _ptr(ws), ws.numel() * ws.element_size(), _stream(),
+                                    upload_stream.cuda_stream, download_stream.cuda_stream)
+    _check(st, "ec_decode_steps_host")

@@ -108,48 +108,26 @@ class ElasticCacheSession:
 
     def compress_host(self, Q_host: torch.Tensor, K_host: torch.Tensor, V_host: torch.Tensor,
                       anchor_pos_host: Optional[torch.Tensor] = None) -> int:
-        """compress() from pinned host tensors. Returns the bytes copied host->device."""
+        """compress() from pinned host tensors (ec_compress_host). Returns the bytes copied host->device."""
         Q, K, V = self._prompt_staging()
-        Q.copy_(Q_host, non_blocking=True)
-        K.copy_(K_host, non_blocking=True)
-        V.copy_(V_host, non_blocking=True)
-        self.compress(Q, K, V)
-        if anchor_pos_host is not None:
-            anchor_pos_host.copy_(self.anchor_pos, non_blocking=True)
+        ec.ec_compress_host(Q_host, K_host, V_host, Q, K, V, self.scores, self.scale, self.n_keep, self.population,
+                            self.protect_ends, self.Kc, self.Vc, self.anchor_pos, anchor_pos_host, self.ws_imp,
+                            self.ws_sel)
+        self.cache = ec.ec_cache_init(self.Kc, self.Vc, self.n_keep, max(self.n_keep, 2),
+                                      min(self.offset, max(self.n_keep, 2) - 1))
         return 3 * Q_host.numel() * Q_host.element_size()
 
     def decode_host(self, q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor,
                     out_host: torch.Tensor, chunk: int = 64):
-        """decode() from pinned host tensors [steps, N, H, D]; writes out_host. Returns (h2d, d2h) bytes.
-
-        The steps are processed in chunks: the upload of the next chunk's inputs and the download of
-        the previous chunk's outputs run on two side streams while the current chunk decodes."""
+        """decode() from pinned host tensors [steps, N, H, D] (ec_decode_steps_host); writes out_host.
+        Returns (h2d, d2h) bytes. Uploads of later chunks and downloads of finished chunks run on two
+        side streams while the current chunk decodes."""
         steps = q_host.shape[0]
+        chunk = max(chunk, -(-steps // 31))                 # the native call takes at most 31 chunks
         q, k, v, out = (t[:steps] for t in self._decode_staging(steps))
-        cur = torch.cuda.current_stream()
         if self._up is None:
             self._up, self._down = torch.cuda.Stream(), torch.cuda.Stream()
-        up, down = self._up, self._down
-        up.wait_stream(cur)                     # staging buffers may still be read by earlier work
-        down.wait_stream(cur)
-        bounds = [(a, min(a + chunk, steps)) for a in range(0, steps, chunk)]
-        ready = []
-        with torch.cuda.stream(up):
-            for a, b in bounds:
-                q[a:b].copy_(q_host[a:b], non_blocking=True)
-                k[a:b].copy_(k_host[a:b], non_blocking=True)
-                v[a:b].copy_(v_host[a:b], non_blocking=True)
-                ev = torch.cuda.Event()
-                ev.record(up)
-                ready.append(ev)
-        for (a, b), ev in zip(bounds, ready):
-            cur.wait_event(ev)
-            self.decode(q[a:b], k[a:b], v[a:b], out[a:b])
-            done = torch.cuda.Event()
-            done.record(cur)
-            with torch.cuda.stream(down):
-                down.wait_event(done)
-                out_host[a:b].copy_(out[a:b], non_blocking=True)
-        cur.wait_stream(down)
+        ec.ec_decode_steps_host(q_host, k_host, v_host, out_host, q, k, v, out, self.cache, self.scale, self.ws_dec,
+                                self._up, self._down, chunk)
         nb = q_host.numel() * q_host.element_size()
         return 3 * nb, nb

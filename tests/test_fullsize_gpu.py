@@ -86,6 +86,13 @@ def test_long_context_units_full_length():
     run_workload(w, [0, 37], [(0, 3), (1, 30)], 40)
 
 
-def test_13b_shapes_full_length_low_ratio():
-    w = wl.WORKLOADS["llava13b_b4"]          # 40 heads, T = 2048, first ratio 0.1 -> 205 kept rows
-    run_workload(w, [3, 150], [(0, 0), (1, 39)], 24)
+@pytest.mark.parametrize("ratio", [0.1, 0.25, 0.5, 0.75])
+def test_13b_shapes_full_length_ratio_sweep(ratio):
+    import dataclasses
+    w = dataclasses.replace(wl.WORKLOADS["llava13b_b4"], keep_ratios=(ratio,))   # 40 heads, T = 2048
+    run_workload(w, [3, 150], [(0, 0), (1, 39)], 20)
+
+
+def test_7b_batch8_shapes_full_length():
+    w = wl.WORKLOADS["llava7b_b8"]           # T = 1024, ratio 0.25 -> 256 kept rows
+    run_workload(w, [0, 100, 255], [(0, 0), (1, 16), (2, 31)], 40)

@@ -594,3 +594,35 @@ def test_second_instruction_on_top_of_a_decoded_cache():
         want, _, _ = queue2.step(qb, kb, vb, scale, policy=orc.POLICY_FIXED, budget=C2, offset=d)
         ec.ec_decode_step(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), nxt.cache, scale, out, nxt.ws_dec)
         assert_bf16_close(out, want, f"decode after the second instruction, step {s}")
+
+
+# ---------------------------------------------------------------- host-resident tensors
+
+def test_host_entry_points_match_the_device_path():
+    """ec_compress_host / ec_decode_steps_host only add copies: same anchors, cache and outputs as the
+    device-resident calls, including a step count that does not divide into whole chunks."""
+    from paper_2407_18121_b200.session import ElasticCacheSession
+    w = wl.WORKLOADS["tiny"]
+    Qb, Kb, Vb = wl.prompt(w)
+    S = 23
+    qb, kb, vb = wl.decode_inputs(w, S)
+    N, H, T, D = Qb.shape
+
+    def pinned(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).pin_memory()
+
+    a = ElasticCacheSession(N, H, T, D, w.keep_ratio, w.offset, w.scale)
+    a.compress(dev_bf16(Qb), dev_bf16(Kb), dev_bf16(Vb))
+    out_a = torch.empty((S, N, H, D), dtype=torch.bfloat16, device="cuda")
+    a.decode(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), out_a)
+
+    b = ElasticCacheSession(N, H, T, D, w.keep_ratio, w.offset, w.scale)
+    anchors_h = torch.full((N, H, b.n_keep), -1, dtype=torch.int32).pin_memory()
+    out_h = torch.zeros((S, N, H, D), dtype=torch.bfloat16).pin_memory()
+    b.compress_host(pinned(Qb), pinned(Kb), pinned(Vb), anchors_h)
+    b.decode_host(pinned(qb), pinned(kb), pinned(vb), out_h, chunk=5)
+    torch.cuda.synchronize()
+    assert torch.equal(a.anchor_pos.cpu(), anchors_h)
+    assert torch.equal(a.Kc, b.Kc) and torch.equal(a.Vc, b.Vc)
+    assert torch.equal(out_a.cpu(), out_h)
+    assert (b.cache.len, b.cache.ring_head, b.cache.step) == (a.cache.len, a.cache.ring_head, a.cache.step)
