@@ -560,7 +560,6 @@ def test_second_instruction_on_top_of_a_decoded_cache():
     sess = ElasticCacheSession(N, H, 2 * C, D, 0.5, d, scale)          # n_keep = C
     assert sess.n_keep == C
     head = S1 % d
-    phys = list(range(C - d)) + [C - d + (i - head) % d for i in range(d)]   # queue position -> slot offset
     Kp, Vp = np.empty_like(Kq), np.empty_like(Vq)
     for pos in range(C):
         slot = pos if pos < C - d else C - d + (head + (pos - (C - d))) % d
