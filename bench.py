@@ -314,6 +314,29 @@ def run_ours(args, w: wl.Workload):
     if status != ec.EC_OK:
         raise SystemExit(f"device status {status}: {ec.status_string(status)}")
 
+    # the same pass recorded once in a CUDA graph and replayed (reported beside the plain launches)
+    graph_ms = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                one_pass()
+        stream.wait_stream(side)
+        for _ in range(2):
+            g.replay()
+        barrier()
+        g0 = torch.cuda.Event(enable_timing=True)
+        g1 = torch.cuda.Event(enable_timing=True)
+        reps = max(1, min(args.steps, 10))
+        g0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        g1.record(stream)
+        barrier()
+        graph_ms = g0.elapsed_time(g1) / reps
+
     # end to end: inputs start in pinned host memory, results are read back every pass
     for _ in range(max(1, min(args.warmup, 2))):
         sess.compress_host(Qh, Kh, Vh, anchors_h)
@@ -362,7 +385,7 @@ def run_ours(args, w: wl.Workload):
         "vs_baseline": None, "dtype": "bf16 storage, fp32 arithmetic", "data": "synthetic",
         "config": workload_config(w),
         "stages_ms": {"importance": imp_ms, "select_merge": mrg_ms, "decode_loop": dec_ms,
-                      "decode_per_token_us": dec_ms * 1e3 / S},
+                      "decode_per_token_us": dec_ms * 1e3 / S, "whole_pass_cuda_graph_replay": graph_ms},
         "decode_only_tokens_per_s": w.batch * S * world / (dec_ms * 1e-3),
         "roofline": {"kernel": "decode_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
@@ -401,6 +424,7 @@ def main():
     ap.add_argument("--oracle-decode-steps", type=int, default=0)
     ap.add_argument("--oracle-problems", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     args = ap.parse_args()
     w = wl.WORKLOADS[args.workload]
     if args.decode_steps:

@@ -625,3 +625,43 @@ def test_host_entry_points_match_the_device_path():
     assert torch.equal(a.Kc, b.Kc) and torch.equal(a.Vc, b.Vc)
     assert torch.equal(out_a.cpu(), out_h)
     assert (b.cache.len, b.cache.ring_head, b.cache.step) == (a.cache.len, a.cache.ring_head, a.cache.step)
+
+
+# ---------------------------------------------------------------- CUDA graph capture of a whole pass
+
+def test_whole_pass_can_be_captured_in_a_cuda_graph_and_replayed():
+    """Every call only enqueues work on the given stream, so a pass (importance, select/merge, decode
+    loop) can be recorded once and replayed. The host-side cache bookkeeping is replayed implicitly:
+    the pass starts from compress(), so each replay sees the same slot sequence."""
+    from paper_2407_18121_b200.session import ElasticCacheSession
+    w = wl.WORKLOADS["tiny"]
+    Qb, Kb, Vb = wl.prompt(w)
+    S = 12
+    qb, kb, vb = wl.decode_inputs(w, S)
+    N, H, T, D = Qb.shape
+    Q, K, V = dev_bf16(Qb), dev_bf16(Kb), dev_bf16(Vb)
+    q, k, v = dev_bf16(qb), dev_bf16(kb), dev_bf16(vb)
+    sess = ElasticCacheSession(N, H, T, D, w.keep_ratio, w.offset, w.scale)
+    out_eager = torch.empty((S, N, H, D), dtype=torch.bfloat16, device="cuda")
+    sess.compress(Q, K, V)                                   # eager reference (also warms everything up)
+    sess.decode(q, k, v, out_eager)
+    torch.cuda.synchronize()
+    Kc_ref, anchors_ref = sess.Kc.clone(), sess.anchor_pos.clone()
+
+    out_graph = torch.zeros_like(out_eager)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            sess.compress(Q, K, V)
+            sess.decode(q, k, v, out_graph)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        out_graph.zero_()
+        sess.Kc.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out_graph, out_eager)
+        assert torch.equal(sess.Kc, Kc_ref) and torch.equal(sess.anchor_pos, anchors_ref)
+    assert ec.ec_device_status(sess.ws_imp) == ec.EC_OK
