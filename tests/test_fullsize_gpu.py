@@ -96,3 +96,52 @@ def test_13b_shapes_full_length_ratio_sweep(ratio):
 def test_7b_batch8_shapes_full_length():
     w = wl.WORKLOADS["llava7b_b8"]           # T = 1024, ratio 0.25 -> 256 kept rows
     run_workload(w, [0, 100, 255], [(0, 0), (1, 16), (2, 31)], 40)
+
+
+def test_longest_supported_prompt():
+    """T = 16384 (the documented maximum), one unit: 128 tiles per pass in the importance kernels,
+    64 KB of keys in the selection kernel's shared memory, 64 slices in the merge kernel."""
+    rng = np.random.default_rng(16384)
+    N, H, T, D, ratio = 1, 1, 16384, 64, 0.1
+    Qb = wl.to_bf16_bits(rng.standard_normal((N, H, T, D)).astype(np.float32))
+    Kb = wl.to_bf16_bits(rng.standard_normal((N, H, T, D)).astype(np.float32))
+    Vb = wl.to_bf16_bits(rng.standard_normal((N, H, T, D)).astype(np.float32))
+    sess = ElasticCacheSession(N, H, T, D, ratio, 16, 0.125)
+    sess.compress(dev_bf16(Qb), dev_bf16(Kb), dev_bf16(Vb))
+    assert ec.ec_device_status(sess.ws_imp) == ec.EC_OK
+    C = sess.n_keep
+    assert C == orc.keep_count(T, ratio) == 1639
+    o_scores, _ = orc.importance(Qb, Kb, 0.125)
+    scores = sess.scores.cpu().double().numpy()
+    assert (np.abs(scores - o_scores) <= SCORE_RTOL * np.abs(o_scores)).all()
+    o_anch = orc.select(o_scores, C, True)
+    anchors = sess.anchor_pos.cpu().numpy()
+    if not (anchors == o_anch).all():
+        s = o_scores[0, 0].copy()
+        s[0] = s[-1] = np.inf
+        kth = np.sort(s)[::-1][C - 1]
+        diff = np.setxor1d(anchors[0, 0], o_anch[0, 0])
+        assert (np.abs(s[diff] - kth) <= 1e-4 * kth).all()
+        o_anch = anchors
+    lo, hi = orc.buckets(o_anch, T)
+    assert close_bf16(host_f64(sess.Kc), orc.merge(Kb, lo, hi)).all()
+    assert close_bf16(host_f64(sess.Vc), orc.merge(Vb, lo, hi)).all()
+
+
+def test_reruns_are_bit_identical():
+    """No kernel uses floating-point atomics or a schedule-dependent reduction order."""
+    w = wl.WORKLOADS["llava7b_b1"]
+    Qb, Kb, Vb = wl.prompt(w, [4, 9])
+    qb, kb, vb = wl.decode_inputs(w, 20, [4, 9])
+    N, H, T, D = Qb.shape
+    Q, K, V, q, k, v = (dev_bf16(x) for x in (Qb, Kb, Vb, qb, kb, vb))
+    results = []
+    for _ in range(2):
+        sess = ElasticCacheSession(N, H, T, D, w.keep_ratio, w.offset, w.scale)
+        sess.compress(Q, K, V)
+        out = torch.empty_like(q)
+        sess.decode(q, k, v, out)
+        torch.cuda.synchronize()
+        results.append((sess.scores.clone(), sess.anchor_pos.clone(), sess.Kc.clone(), sess.Vc.clone(), out))
+    for a, b in zip(*results):
+        assert torch.equal(a, b)
