@@ -31,6 +31,7 @@ constexpr int kTmemCols = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s per wait, then give up
+constexpr unsigned kPollBackoffNs = 32;                      // sleep between polls of the TMA / MMA threads
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -68,12 +69,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
 
 // Bounded wait. Returns false when the CTA is aborting or the time limit passed (in which
 // case the abort flag and the global status word are set).
+// `backoff_ns` > 0 makes the poller sleep between attempts: used by the single-thread TMA and MMA
+// roles so that their polling does not take issue slots from the softmax warps of the same SM.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                          unsigned long long limit_ns = kWaitLimitNs)
+                                          unsigned long long limit_ns = kWaitLimitNs, unsigned backoff_ns = 0)
 {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t spin = 1;; ++spin) {
+        if (backoff_ns) __nanosleep(backoff_ns);
         if (mbar_try(bar, parity)) return true;
         if ((spin & 63u) == 0) {
             if (*abort_flag) return false;
@@ -293,14 +297,14 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     int unit, st, first, count;
                     if (!item_of(sidx, sub, unit, st, first, count)) break;
                     // the stationary buffer is free once the previous item's last MMA has completed
-                    if (!mbar_wait(bar_stat_empty, (it + 1u) & 1u, abort_flag, status)) { alive = false; break; }
+                    if (!mbar_wait(bar_stat_empty, (it + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                     mbar_expect_tx(bar_stat_full, kTileBytes);
 #pragma unroll
                     for (int bx = 0; bx < kBoxes; ++bx)
                         tma_load_3d(base + L::kStat + bx * kBoxBytes, map_stat, bx * 64, st * kTileRows, unit, bar_stat_full);
                     for (int t = 0; t < count; ++t, ++tg) {
                         const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
-                        if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, status)) { alive = false; break; }
+                        if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                         mbar_expect_tx(bar_full(s), kTileBytes);
 #pragma unroll
                         for (int bx = 0; bx < kBoxes; ++bx)
@@ -325,12 +329,12 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 for (int sub = 0; alive && sub < 2; ++sub) {
                     int unit, st, first, count;
                     if (!item_of(sidx, sub, unit, st, first, count)) break;
-                    if (!mbar_wait(bar_stat_full, it & 1u, abort_flag, status)) { alive = false; break; }
+                    if (!mbar_wait(bar_stat_full, it & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                     for (int t = 0; t < count; ++t, ++tg) {
                         const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
                         const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
-                        if (!mbar_wait(bar_acc_empty(b), bph ^ 1u, abort_flag, status)) { alive = false; break; }
-                        if (!mbar_wait(bar_full(s), ph, abort_flag, status)) { alive = false; break; }
+                        if (!mbar_wait(bar_acc_empty(b), bph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                        if (!mbar_wait(bar_full(s), ph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                         tc_fence_after();
                         const uint32_t a0 = base + L::kStat, b0 = base + L::kStage0 + s * kTileBytes;
 #pragma unroll
@@ -389,9 +393,10 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) if (i > lim) v[i] = -INFINITY;
                             }
-                            float cm = v[0];
+                            float cm4[4] = {v[0], v[1], v[2], v[3]};      // four chains instead of one of 31
 #pragma unroll
-                            for (int i = 1; i < 32; ++i) cm = fmaxf(cm, v[i]);
+                            for (int i = 4; i < 32; ++i) cm4[i & 3] = fmaxf(cm4[i & 3], v[i]);
+                            const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
                             const float mnew = fmaxf(mrun, cm * c);
                             if (mnew != -INFINITY) {
                                 float part[4] = {0.f, 0.f, 0.f, 0.f};
