@@ -25,7 +25,7 @@ namespace ec {
 namespace {
 
 constexpr int kTileRows = 128;            // rows of a tile = MMA M = MMA N
-constexpr int kThreads = 192;             // 6 warps: TMA, MMA, 4 x softmax
+constexpr int kThreads = 320;             // 10 warps: TMA, MMA, 8 x softmax (two per TMEM lane quarter)
 constexpr int kAccBufs = 2;               // TMEM accumulator buffers (128 columns each)
 constexpr int kTmemCols = 256;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -187,10 +187,11 @@ struct Smem {
     static constexpr int kStat = 0;
     static constexpr int kStage0 = kTileBytes;
     static constexpr int kLse = kStage0 + STAGES * kTileBytes;            // 2 x 128 floats
-    static constexpr int kBars = kLse + kAccBufs * kTileRows * 4;
+    static constexpr int kComb = kLse + kAccBufs * kTileRows * 4;         // 128 x float2: half-row results
+    static constexpr int kBars = kComb + kTileRows * 8;
     // barrier slots (8 bytes each): stat_full, stat_empty, full[STAGES], empty[STAGES],
-    // acc_full[2], acc_empty[2], lse_ready[2]
-    static constexpr int kNumBars = 2 + 2 * STAGES + 3 * kAccBufs;
+    // acc_full[2], acc_empty[2], lse_ready[2], comb_full, comb_empty
+    static constexpr int kNumBars = 2 + 2 * STAGES + 3 * kAccBufs + 2;
     static constexpr int kTmemSlot = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemSlot + 4;
     static constexpr int kTotal = kAbort + 4;
@@ -233,6 +234,9 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     auto bar_acc_full = [&](int b) { return bars + 8u * (2 + 2 * STAGES + b); };
     auto bar_acc_empty = [&](int b) { return bars + 8u * (2 + 2 * STAGES + kAccBufs + b); };
     auto bar_lse = [&](int b) { return bars + 8u * (2 + 2 * STAGES + 2 * kAccBufs + b); };
+    const uint32_t bar_comb_full = bars + 8u * (2 + 2 * STAGES + 3 * kAccBufs);
+    const uint32_t bar_comb_empty = bar_comb_full + 8u;
+    float2 *comb_s = reinterpret_cast<float2 *>(base_ptr + L::kComb);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + L::kTmemSlot);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + L::kAbort);
     float *lse_s = reinterpret_cast<float *>(base_ptr + L::kLse);
@@ -254,9 +258,11 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(bar_acc_full(b), 1);
-            mbar_init(bar_acc_empty(b), 4);
+            mbar_init(bar_acc_empty(b), 8);
             mbar_init(bar_lse(b), 4 * 32);
         }
+        mbar_init(bar_comb_full, 4 * 32);
+        mbar_init(bar_comb_empty, 4 * 32);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -353,9 +359,13 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
     } else {
         // ---------------------------------------------------------------- softmax warps
+        // Two warps share each TMEM lane quarter: warps 2..5 take columns 0..63 of a tile, warps
+        // 6..9 columns 64..127. A row's two half results meet through shared memory at the end of
+        // an item. Eight warps instead of four keep the ex2 pipe fed while others wait on TMEM.
         const int q4 = warp & 3;                              // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                     // which 64 columns of every tile
         const int r = q4 * 32 + lane;                         // row of the stationary tile = TMEM lane
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(half * 64);
         const int Tk = geo.Tk();
         for (int sidx = blockIdx.x; alive && sidx < n_super; sidx += gridDim.x) {
             for (int sub = 0; alive && sub < 2; ++sub) {
@@ -373,16 +383,19 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     const int off = (PASS2 ? tile - st : st - tile) * kTileRows + geo.P;
                     const bool masked = off < kTileRows - 1;
                     if (PASS2) {
-                        // every softmax thread stages one entry of the tile's lse, then all wait (bounded)
-                        // for the 128 entries; the buffer is reused two tiles later, after the next
-                        // tile's rendezvous
-                        lse_s[b * kTileRows + r] = lse2[lse_row + (size_t)tile * kTileRows + r];
-                        mbar_arrive(bar_lse(b));
+                        // the first-half threads stage one entry each of the tile's lse, then all wait
+                        // (bounded) for the 128 entries; the buffer is reused two tiles later, after the
+                        // next tile's rendezvous
+                        if (half == 0) {
+                            lse_s[b * kTileRows + r] = lse2[lse_row + (size_t)tile * kTileRows + r];
+                            mbar_arrive(bar_lse(b));
+                        }
                         if (!mbar_wait(bar_lse(b), bph, abort_flag, status)) { alive = false; break; }
                     }
                     if (!mbar_wait(bar_acc_full(b), bph, abort_flag, status)) { alive = false; break; }
                     tc_fence_after();
 
+                    // `ch` = index of the 32-column chunk inside the 128-column tile
                     auto chunk = [&](uint32_t (&raw)[32], int ch) {
                         float v[32];
 #pragma unroll
@@ -425,33 +438,41 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         }
                     };
 
-                    // the load of the next 32 columns is in flight while the current ones are processed
+                    // this thread's 64 columns: the second 32 are in flight while the first are processed
                     const uint32_t col0 = lane_addr + b * kTileRows;
                     uint32_t ra[32], rb[32];
                     tmem_ld32_async(col0, ra);
                     tmem_ld_wait(ra);
                     tmem_ld32_async(col0 + 32, rb);
-                    chunk(ra, 0);
-                    tmem_ld_wait(rb);
-                    tmem_ld32_async(col0 + 64, ra);
-                    chunk(rb, 1);
-                    tmem_ld_wait(ra);
-                    tmem_ld32_async(col0 + 96, rb);
-                    chunk(ra, 2);
+                    chunk(ra, half * 2);
                     tmem_ld_wait(rb);
                     tc_fence_before();                   // all TMEM reads of this tile are done:
                     __syncwarp();                        // hand the accumulator back before the last chunk's math
                     if (lane == 0) mbar_arrive(bar_acc_empty(b));
-                    chunk(rb, 3);
+                    chunk(rb, half * 2 + 1);
                 }
                 if (!alive) break;
-                const int row = st * kTileRows + r;
-                if (!PASS2) {
-                    const float l2 = (row < geo.Tq) ? mrun + __log2f(Z) : INFINITY;
-                    lse2[lse_row + row] = l2;
-                    if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
-                } else if (row < Tk) {
-                    scores[(size_t)unit * Tk + row] = (acc0 + acc1) + (acc2 + acc3);
+
+                // the two halves of a row meet: the second-half thread hands its result over
+                const uint32_t iph = it & 1u;
+                if (half == 1) {
+                    if (!mbar_wait(bar_comb_empty, iph ^ 1u, abort_flag, status)) { alive = false; break; }
+                    comb_s[r] = PASS2 ? make_float2((acc0 + acc1) + (acc2 + acc3), 0.f) : make_float2(mrun, Z);
+                    mbar_arrive(bar_comb_full);
+                } else {
+                    if (!mbar_wait(bar_comb_full, iph, abort_flag, status)) { alive = false; break; }
+                    const float2 o = comb_s[r];
+                    mbar_arrive(bar_comb_empty);
+                    const int row = st * kTileRows + r;
+                    if (!PASS2) {
+                        const float M = fmaxf(mrun, o.x);             // finite: column 0 of some tile is visible
+                        const float Zs = Z * fast_exp2(mrun - M) + o.y * fast_exp2(o.x - M);
+                        const float l2 = (row < geo.Tq) ? M + __log2f(Zs) : INFINITY;
+                        lse2[lse_row + row] = l2;
+                        if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
+                    } else if (row < Tk) {
+                        scores[(size_t)unit * Tk + row] = ((acc0 + acc1) + (acc2 + acc3)) + o.x;
+                    }
                 }
                 ++it;
             }
