@@ -374,6 +374,8 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const size_t lse_row = (size_t)unit * geo.ntq * kTileRows;
                 float mrun = -INFINITY, Z = 0.f;                      // pass 1 running max / sum (log2 domain)
                 float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f; // pass 2 column sum
+                float lse_ahead = 0.f;
+                if (PASS2 && half == 0) lse_ahead = lse2[lse_row + (size_t)first * kTileRows + r];
                 for (int t = 0; t < count; ++t, ++tg) {
                     const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
                     const int tile = stream_tile(first, t);
@@ -383,12 +385,15 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     const int off = (PASS2 ? tile - st : st - tile) * kTileRows + geo.P;
                     const bool masked = off < kTileRows - 1;
                     if (PASS2) {
-                        // the first-half threads stage one entry each of the tile's lse, then all wait
+                        // the first-half threads stage one entry each of the tile's lse (fetched one tile
+                        // ahead, so its latency hides behind the previous tile's math), then all wait
                         // (bounded) for the 128 entries; the buffer is reused two tiles later, after the
                         // next tile's rendezvous
                         if (half == 0) {
-                            lse_s[b * kTileRows + r] = lse2[lse_row + (size_t)tile * kTileRows + r];
+                            lse_s[b * kTileRows + r] = lse_ahead;
                             mbar_arrive(bar_lse(b));
+                            if (t + 1 < count)
+                                lse_ahead = lse2[lse_row + (size_t)stream_tile(first, t + 1) * kTileRows + r];
                         }
                         if (!mbar_wait(bar_lse(b), bph, abort_flag, status)) { alive = false; break; }
                     }
