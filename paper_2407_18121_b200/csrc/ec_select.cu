@@ -45,53 +45,89 @@ select_kernel(const float *__restrict__ scores, int T, int C, int protect_ends, 
     const size_t unit = blockIdx.x;
     const float *s = scores + unit * T;
 
+    // Protected positions (first and last) are always anchors: they get the top key and are left
+    // out of the search for the threshold among the others.
+    auto is_prot = [&](int t) { return protect_ends && (t == 0 || (t == T - 1 && C >= 2)); };
+    const int nprot = protect_ends ? ((C >= 2 && T >= 2) ? 2 : 1) : 0;
+    const uint32_t need0 = (uint32_t)(C - nprot);        // anchors still to find among unprotected keys
+
+    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
     for (int t = tid; t < T; t += kSelThreads) {
         uint32_t k = sort_key(s[t]);
-        if (protect_ends && (t == 0 || (t == T - 1 && C >= 2))) k = 0xFFFFFFFFu;
+        if (is_prot(t)) k = 0xFFFFFFFFu;
+        else { kmin = min(kmin, k); kmax = max(kmax, k); }
         keys[t] = k;
     }
-    if (tid == 0) { s_prefix = 0; s_need = (uint32_t)C; }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
+        kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
+    }
+    if ((tid & 31) == 0) { warp_gt[tid >> 5] = kmin; warp_eq[tid >> 5] = kmax; }   // reused below for the scan
+    __syncthreads();
+    kmin = warp_gt[0];
+    kmax = warp_eq[0];
+#pragma unroll
+    for (int w = 1; w < kSelThreads / 32; ++w) { kmin = min(kmin, warp_gt[w]); kmax = max(kmax, warp_eq[w]); }
     __syncthreads();
 
-    // Four 8-bit digits, most significant first: find the C-th largest key.
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        hist[tid] = 0;                       // kSelThreads == 256 bins
-        __syncthreads();
-        const uint32_t prefix = s_prefix, need = s_need;
-        const uint32_t himask = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
-        for (int t = tid; t < T; t += kSelThreads) {
-            uint32_t k = keys[t];
-            if ((k & himask) == prefix) atomicAdd(&hist[(k >> shift) & 0xFF], 1u);
+    // Radix select for the need0-th largest unprotected key. All keys agree on the bits above the
+    // highest bit in which the smallest and the largest key differ, so only the bits below it are
+    // examined, 8 at a time from the top: the digits spread over the keys' real range (attention
+    // column sums lie within a few octaves, so a fixed top byte would put them all in a few bins).
+    if (need0 == 0) {
+        if (tid == 0) { s_prefix = 0xFFFFFFFEu; s_need = 0; }             // only the protected keys pass
+    } else if (kmin == kmax) {
+        if (tid == 0) { s_prefix = kmin; s_need = need0; }                // every key is a tie
+    } else {
+        const int nbits = 32 - __clz(kmin ^ kmax);                        // bits that vary: [nbits-1 .. 0]
+        const int passes = (nbits + 7) / 8;
+        if (tid == 0) {
+            s_prefix = (nbits == 32) ? 0u : (kmax >> nbits) << nbits;     // the common high bits
+            s_need = need0;
         }
-        __syncthreads();
-        if (tid < 32) {
-            // lane l owns bins 255-8l .. 248-8l (descending); suffix-scan across lanes
-            uint32_t local[8], sum = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { local[i] = hist[255 - (tid * 8 + i)]; sum += local[i]; }
-            uint32_t incl = sum;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                if (tid >= o) incl += v;
+        for (int pass = 0; pass < passes; ++pass) {
+            const int shift = 8 * (passes - 1 - pass);
+            const int width = (pass == 0) ? nbits - shift : 8;            // the top digit may be narrower
+            const uint32_t dmask = (1u << width) - 1u;
+            const uint32_t himask = (shift + width >= 32) ? 0u : (0xFFFFFFFFu << (shift + width));
+            hist[tid] = 0;                       // kSelThreads == 256 bins
+            __syncthreads();
+            const uint32_t prefix = s_prefix, need = s_need;
+            for (int t = tid; t < T; t += kSelThreads) {
+                const uint32_t k = keys[t];
+                if ((k & himask) == (prefix & himask) && !is_prot(t)) atomicAdd(&hist[(k >> shift) & dmask], 1u);
             }
-            uint32_t before = incl - sum;    // keys in strictly higher bins than this lane's
-            if (before < need && need <= incl) {
-                uint32_t run = before;
+            __syncthreads();
+            if (tid < 32) {
+                // lane l owns bins 255-8l .. 248-8l (descending); suffix-scan across lanes
+                uint32_t local[8], sum = 0;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (run < need && need <= run + local[i]) {
-                        s_prefix = prefix | ((uint32_t)(255 - (tid * 8 + i)) << shift);
-                        s_need = need - run;  // how many are still needed inside this bin
+                for (int i = 0; i < 8; ++i) { local[i] = hist[255 - (tid * 8 + i)]; sum += local[i]; }
+                uint32_t incl = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (tid >= o) incl += v;
+                }
+                uint32_t before = incl - sum;    // keys in strictly higher bins than this lane's
+                if (before < need && need <= incl) {
+                    uint32_t run = before;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (run < need && need <= run + local[i]) {
+                            s_prefix = prefix | ((uint32_t)(255 - (tid * 8 + i)) << shift);
+                            s_need = need - run;  // how many are still needed inside this bin
+                        }
+                        run += local[i];
                     }
-                    run += local[i];
                 }
             }
+            __syncthreads();
         }
-        __syncthreads();
     }
-    const uint32_t thr = s_prefix;       // key of the C-th largest element
+    __syncthreads();
+    const uint32_t thr = s_prefix;       // key of the last anchor taken by score (protected keys lie above it)
     const uint32_t need_eq = s_need;     // how many keys equal to thr are taken (lowest positions)
 
     // Ordered compaction: thread i owns the contiguous positions [i*ipt, (i+1)*ipt).
