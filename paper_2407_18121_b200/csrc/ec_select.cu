@@ -1,12 +1,11 @@
-// Anchor selection (Sec. 3.3: the N_I positions with the highest importance, ascending)
-// as an exact radix select on fp32 bit patterns followed by an order-preserving compaction.
+// Anchor selection (Sec. 3.3: the N_I positions with the highest importance, ascending):
+// a warp-level radix select over bit planes held in registers finds the exact N_I-th largest fp32
+// bit pattern, then warp ballots list the anchors in position order.
 #include "ec_common.cuh"
 
 namespace ec {
 
 namespace {
-
-constexpr int kSelThreads = 256;
 
 // Order-preserving map from fp32 to uint32 (larger float -> larger key).
 __device__ __forceinline__ uint32_t sort_key(float x)
@@ -28,179 +27,211 @@ __global__ void group_mean_kernel(const float *__restrict__ scores, float *__res
     mean[grp * T + t] = acc / (float)share;
 }
 
-// One CTA per selection unit. Dynamic shared memory: T keys + n_keep anchors.
-// `replicate` > 1 writes the same anchors for that many consecutive heads (layer-shared mode).
-__global__ void __launch_bounds__(kSelThreads)
-select_kernel(const float *__restrict__ scores, int T, int C, int protect_ends, int replicate,
+constexpr int kKeysPerLane = 32;                        // a warp holds 1024 consecutive positions
+constexpr int kWarpSpan = 32 * kKeysPerLane;
+constexpr int kMaxWarpsPerUnit = 16;                    // T <= 16384
+
+// In-register transpose of a 32 x 32 bit matrix (row i = word a[i], column c = bit 31 - c):
+// five butterfly stages of masked swaps between words.
+__device__ __forceinline__ void transpose32(uint32_t (&a)[32])
+{
+    uint32_t m = 0x0000FFFFu;
+#pragma unroll
+    for (int j = 16; j != 0; j >>= 1) {
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            if ((k & j) == 0) {
+                const uint32_t t = (a[k] ^ (a[k + j] >> j)) & m;
+                a[k] ^= t;
+                a[k + j] ^= t << j;
+            }
+        }
+        m ^= m << (j >> 1);
+    }
+}
+
+// Warp-level selection. G warps share one unit (G = ceil(T / 1024)); with G == 1 a CTA holds four
+// independent units, one per warp, and no block-wide barrier is ever needed. Lane l of warp w owns
+// positions 1024*w + 32*j + l (j = 0..31, its "rows").
+//  1. The lane's 32 keys (order-preserving uint32 images of the scores) are transposed into 32
+//     bit planes, so "how many of my still-undecided keys have bit b set" is one AND and one popc.
+//  2. Radix descent from the top bit for the C-th largest key: if at least `need` undecided keys of
+//     the unit have the bit set, those stay undecided and the others are out; otherwise they are all
+//     anchors (`greater`), `need` shrinks by their count and the others stay undecided. All keys
+//     agree on the bits above the highest bit in which the smallest and the largest key differ, so
+//     the descent starts there. What is still undecided at the end equals the threshold: ties, of
+//     which the `need` lowest positions are taken. Protected positions (first, last) are anchors
+//     from the start.
+//  3. Ordered compaction with warp ballots, one row of 32 consecutive positions at a time.
+// `replicate` > 1 writes the same anchors for that many consecutive heads (shared populations).
+template <int G>
+__global__ void __launch_bounds__(G == 1 ? 128 : 32 * G)
+select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int protect_ends, int replicate,
               int32_t *__restrict__ anchor_pos, int32_t *__restrict__ bucket_len)
 {
-    extern __shared__ uint32_t smem[];
-    uint32_t *keys = smem;
-    int32_t *anch = reinterpret_cast<int32_t *>(smem + T);
-    __shared__ uint32_t hist[256];
-    __shared__ uint32_t s_prefix, s_need;
-    __shared__ uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32];
+    __shared__ uint32_t xa[2][kMaxWarpsPerUnit], xb[kMaxWarpsPerUnit];     // cross-warp exchange (G > 1)
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int unit = (G == 1) ? blockIdx.x * 4 + warp : blockIdx.x;
+    if (G == 1 && unit >= n_units) return;                 // whole warp leaves; no barriers in this variant
+    const int wu = (G == 1) ? 0 : warp;                    // this warp's index inside the unit
+    const int base = wu * kWarpSpan;
+    const float *s = scores + (size_t)unit * T;
 
-    const int tid = threadIdx.x;
-    const size_t unit = blockIdx.x;
-    const float *s = scores + unit * T;
-
-    // Protected positions (first and last) are always anchors: they get the top key and are left
-    // out of the search for the threshold among the others.
     auto is_prot = [&](int t) { return protect_ends && (t == 0 || (t == T - 1 && C >= 2)); };
     const int nprot = protect_ends ? ((C >= 2 && T >= 2) ? 2 : 1) : 0;
-    const uint32_t need0 = (uint32_t)(C - nprot);        // anchors still to find among unprotected keys
+    int par = 0;
+    auto unit_sum = [&](uint32_t v) {                      // sum over the unit's warps, same value in every thread
+        v = __reduce_add_sync(0xFFFFFFFFu, v);
+        if (G == 1) return v;
+        if (lane == 0) xa[par][wu] = v;
+        __syncthreads();                                   // buffers alternate: one barrier per use
+        uint32_t t = 0;
+#pragma unroll
+        for (int w = 0; w < G; ++w) t += xa[par][w];
+        par ^= 1;
+        return t;
+    };
 
-    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-    for (int t = tid; t < T; t += kSelThreads) {
-        uint32_t k = sort_key(s[t]);
-        if (is_prot(t)) k = 0xFFFFFFFFu;
-        else { kmin = min(kmin, k); kmax = max(kmax, k); }
-        keys[t] = k;
+    // a[31 - j] = key of row j, so that after the transpose a[31 - b] is the plane of key bit b with
+    // row j at mask bit j
+    uint32_t a[32];
+    uint32_t undecided = 0u, greater = 0u;                 // row masks
+    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;               // range of the unprotected keys
+#pragma unroll
+    for (int j = 0; j < kKeysPerLane; ++j) {               // all loads first, so that they overlap
+        const int t = base + 32 * j + lane;
+        a[31 - j] = (t < T) ? __float_as_uint(__ldg(s + t)) : 0u;
     }
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) {
-        kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
-        kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
-    }
-    if ((tid & 31) == 0) { warp_gt[tid >> 5] = kmin; warp_eq[tid >> 5] = kmax; }   // reused below for the scan
-    __syncthreads();
-    kmin = warp_gt[0];
-    kmax = warp_eq[0];
-#pragma unroll
-    for (int w = 1; w < kSelThreads / 32; ++w) { kmin = min(kmin, warp_gt[w]); kmax = max(kmax, warp_eq[w]); }
-    __syncthreads();
-
-    // Radix select for the need0-th largest unprotected key. All keys agree on the bits above the
-    // highest bit in which the smallest and the largest key differ, so only the bits below it are
-    // examined, 8 at a time from the top: the digits spread over the keys' real range (attention
-    // column sums lie within a few octaves, so a fixed top byte would put them all in a few bins).
-    if (need0 == 0) {
-        if (tid == 0) { s_prefix = 0xFFFFFFFEu; s_need = 0; }             // only the protected keys pass
-    } else if (kmin == kmax) {
-        if (tid == 0) { s_prefix = kmin; s_need = need0; }                // every key is a tie
-    } else {
-        const int nbits = 32 - __clz(kmin ^ kmax);                        // bits that vary: [nbits-1 .. 0]
-        const int passes = (nbits + 7) / 8;
-        if (tid == 0) {
-            s_prefix = (nbits == 32) ? 0u : (kmax >> nbits) << nbits;     // the common high bits
-            s_need = need0;
+    for (int j = 0; j < kKeysPerLane; ++j) {
+        const int t = base + 32 * j + lane;
+        uint32_t key = 0u;
+        if (t < T) {
+            key = sort_key(__uint_as_float(a[31 - j]));
+            if (is_prot(t)) greater |= 1u << j;
+            else { undecided |= 1u << j; kmin = min(kmin, key); kmax = max(kmax, key); }
         }
-        for (int pass = 0; pass < passes; ++pass) {
-            const int shift = 8 * (passes - 1 - pass);
-            const int width = (pass == 0) ? nbits - shift : 8;            // the top digit may be narrower
-            const uint32_t dmask = (1u << width) - 1u;
-            const uint32_t himask = (shift + width >= 32) ? 0u : (0xFFFFFFFFu << (shift + width));
-            hist[tid] = 0;                       // kSelThreads == 256 bins
-            __syncthreads();
-            const uint32_t prefix = s_prefix, need = s_need;
-            for (int t = tid; t < T; t += kSelThreads) {
-                const uint32_t k = keys[t];
-                if ((k & himask) == (prefix & himask) && !is_prot(t)) atomicAdd(&hist[(k >> shift) & dmask], 1u);
-            }
-            __syncthreads();
-            if (tid < 32) {
-                // lane l owns bins 255-8l .. 248-8l (descending); suffix-scan across lanes
-                uint32_t local[8], sum = 0;
+        a[31 - j] = key;
+    }
+    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+    if (G > 1) {
+        if (lane == 0) { xa[par][wu] = kmin; xb[wu] = kmax; }
+        __syncthreads();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { local[i] = hist[255 - (tid * 8 + i)]; sum += local[i]; }
-                uint32_t incl = sum;
+        for (int w = 0; w < G; ++w) { kmin = min(kmin, xa[par][w]); kmax = max(kmax, xb[w]); }
+        par ^= 1;
+    }
+    transpose32(a);
+
+    uint32_t need = (uint32_t)(C - nprot);                // anchors still to find among the unprotected keys
+    if (need == 0) {
+        undecided = 0u;                                   // only the protected keys are anchors
+    } else if (kmin != kmax) {                            // (kmin == kmax: every unprotected key is a tie)
+        const int nbits = 32 - __clz(kmin ^ kmax);
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                    if (tid >= o) incl += v;
-                }
-                uint32_t before = incl - sum;    // keys in strictly higher bins than this lane's
-                if (before < need && need <= incl) {
-                    uint32_t run = before;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        if (run < need && need <= run + local[i]) {
-                            s_prefix = prefix | ((uint32_t)(255 - (tid * 8 + i)) << shift);
-                            s_need = need - run;  // how many are still needed inside this bin
-                        }
-                        run += local[i];
-                    }
+        for (int b = 31; b >= 0; --b) {
+            if (b < nbits) {                              // uniform over the unit
+                const uint32_t ones = undecided & a[31 - b];
+                const uint32_t c1 = unit_sum(__popc(ones));
+                if (c1 >= need) {
+                    undecided = ones;
+                } else {
+                    need -= c1;
+                    greater |= ones;
+                    undecided &= ~a[31 - b];
                 }
             }
-            __syncthreads();
         }
     }
-    __syncthreads();
-    const uint32_t thr = s_prefix;       // key of the last anchor taken by score (protected keys lie above it)
-    const uint32_t need_eq = s_need;     // how many keys equal to thr are taken (lowest positions)
+    const uint32_t need_eq = need;                        // ties taken, lowest positions first
 
-    // Ordered compaction: thread i owns the contiguous positions [i*ipt, (i+1)*ipt).
-    const int ipt = (T + kSelThreads - 1) / kSelThreads;
-    const int t0 = min(tid * ipt, T), t1 = min(t0 + ipt, T);
-    uint32_t gt = 0, eq = 0;
-    for (int t = t0; t < t1; ++t) {
-        uint32_t k = keys[t];
-        gt += (k > thr);
-        eq += (k == thr);
-    }
-    uint32_t gt_incl = gt, eq_incl = eq;
-    const int lane = tid & 31, warp = tid >> 5;
+    // anchors / ties held by earlier warps of the unit
+    uint32_t gb = 0, eb = 0;
+    if (G > 1) {
+        const uint32_t gt = __reduce_add_sync(0xFFFFFFFFu, __popc(greater));
+        const uint32_t eq = __reduce_add_sync(0xFFFFFFFFu, __popc(undecided));
+        if (lane == 0) { xa[par][wu] = gt; xb[wu] = eq; }
+        __syncthreads();
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        uint32_t a = __shfl_up_sync(0xFFFFFFFFu, gt_incl, o);
-        uint32_t b = __shfl_up_sync(0xFFFFFFFFu, eq_incl, o);
-        if (lane >= o) { gt_incl += a; eq_incl += b; }
+        for (int w = 0; w < G; ++w)
+            if (w < wu) { gb += xa[par][w]; eb += xb[w]; }
+        par ^= 1;
     }
-    if (lane == 31) { warp_gt[warp] = gt_incl; warp_eq[warp] = eq_incl; }
-    __syncthreads();
-    uint32_t gt_before = gt_incl - gt, eq_before = eq_incl - eq;
-    for (int w = 0; w < warp; ++w) { gt_before += warp_gt[w]; eq_before += warp_eq[w]; }
-    for (int t = t0; t < t1; ++t) {
-        uint32_t k = keys[t];
-        if (k > thr) {
-            anch[gt_before + min(eq_before, need_eq)] = t;
-            ++gt_before;
-        } else if (k == thr) {
-            if (eq_before < need_eq) anch[gt_before + eq_before] = t;
-            ++eq_before;
+
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    int32_t *ap0 = anchor_pos + (size_t)unit * replicate * C;
+#pragma unroll
+    for (int j = 0; j < kKeysPerLane; ++j) {
+        const bool is_gt = (greater >> j) & 1u, is_eq = (undecided >> j) & 1u;
+        const uint32_t bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
+        const uint32_t g_here = gb + __popc(bg & lt_mask), e_here = eb + __popc(be & lt_mask);
+        int idx = -1;                                      // anchors before this position = its own index
+        if (is_gt) idx = (int)(g_here + min(e_here, need_eq));
+        else if (is_eq && e_here < need_eq) idx = (int)(g_here + e_here);
+        if (idx >= 0) {
+            const int t = base + 32 * j + lane;
+            for (int r = 0; r < replicate; ++r) ap0[(size_t)r * C + idx] = t;
         }
+        gb += __popc(bg);
+        eb += __popc(be);
     }
-    __syncthreads();
 
     // the merge kernel behind this one may start scheduling; it waits for this grid to finish
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    for (int r = 0; r < replicate; ++r) {
-        int32_t *ap = anchor_pos + (unit * replicate + r) * C;
-        for (int k = tid; k < C; k += kSelThreads) ap[k] = anch[k];
-        if (bucket_len) {
-            // Eq. 2: bucket k spans floor((t_{k-1}+t_k)/2)+1 .. floor((t_k+t_{k+1})/2)
-            int32_t *bl = bucket_len + (unit * replicate + r) * C;
-            for (int k = tid; k < C; k += kSelThreads) {
-                int lo = (k == 0) ? 0 : ((anch[k - 1] + anch[k]) >> 1) + 1;
-                int hi = (k == C - 1) ? T - 1 : ((anch[k] + anch[k + 1]) >> 1);
-                bl[k] = hi - lo + 1;
-            }
+    if (bucket_len) {
+        // Eq. 2: bucket k spans floor((t_{k-1}+t_k)/2)+1 .. floor((t_k+t_{k+1})/2); the anchors just
+        // written by the unit's own warps are visible after the barrier
+        if (G == 1) __syncwarp(); else __syncthreads();
+        const volatile int32_t *av = ap0;
+        for (int kk = wu * 32 + lane; kk < C; kk += 32 * G) {
+            const int c0 = av[kk];
+            const int lo = (kk == 0) ? 0 : ((av[kk - 1] + c0) >> 1) + 1;
+            const int hi = (kk == C - 1) ? T - 1 : ((c0 + av[kk + 1]) >> 1);
+            for (int r = 0; r < replicate; ++r) bucket_len[((size_t)unit * replicate + r) * C + kk] = hi - lo + 1;
         }
     }
 }
 
 }  // namespace
 
+namespace {
+template <int G>
+cudaError_t launch_select_t(const float *scores, int n_units, int T, int n_keep, int protect_ends, int replicate,
+                            int32_t *anchor_pos, int32_t *bucket_len, cudaStream_t stream)
+{
+    const unsigned grid = (G == 1) ? (unsigned)((n_units + 3) / 4) : (unsigned)n_units;
+    select_kernel<G><<<grid, G == 1 ? 128 : 32 * G, 0, stream>>>(scores, n_units, T, n_keep, protect_ends, replicate,
+                                                                 anchor_pos, bucket_len);
+    return cudaGetLastError();
+}
+}  // namespace
+
 // `share` consecutive units rank one common (averaged) score vector; share == 1: every unit its own.
 cudaError_t launch_select(const float *scores, int units, int T, int n_keep, int share, int protect_ends,
                           int32_t *anchor_pos, int32_t *bucket_len, float *mean_ws, cudaStream_t stream)
 {
-    size_t smem = (size_t)(T + n_keep) * sizeof(uint32_t);
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    const float *src = scores;
+    int n = units, rep = 1;
     if (share > 1) {
         const int groups = units / share;
         if (groups > 65535) return cudaErrorInvalidConfiguration;
         dim3 g((T + 255) / 256, groups);
         group_mean_kernel<<<g, 256, 0, stream>>>(scores, mean_ws, share, T);
-        select_kernel<<<groups, kSelThreads, smem, stream>>>(mean_ws, T, n_keep, protect_ends, share, anchor_pos, bucket_len);
-    } else {
-        select_kernel<<<units, kSelThreads, smem, stream>>>(scores, T, n_keep, protect_ends, 1, anchor_pos, bucket_len);
+        src = mean_ws;
+        n = groups;
+        rep = share;
     }
-    return cudaGetLastError();
+    const int G = (T + kWarpSpan - 1) / kWarpSpan;
+    switch (G) {
+    case 1: return launch_select_t<1>(src, n, T, n_keep, protect_ends, rep, anchor_pos, bucket_len, stream);
+    case 2: return launch_select_t<2>(src, n, T, n_keep, protect_ends, rep, anchor_pos, bucket_len, stream);
+    case 3: case 4: return launch_select_t<4>(src, n, T, n_keep, protect_ends, rep, anchor_pos, bucket_len, stream);
+    case 5: case 6: case 7: case 8: return launch_select_t<8>(src, n, T, n_keep, protect_ends, rep, anchor_pos, bucket_len, stream);
+    default: break;
+    }
+    if (G > kMaxWarpsPerUnit) return cudaErrorInvalidConfiguration;
+    return launch_select_t<16>(src, n, T, n_keep, protect_ends, rep, anchor_pos, bucket_len, stream);
 }
 
 }  // namespace ec
