@@ -31,22 +31,24 @@ constexpr int kKeysPerLane = 32;                        // a warp holds 1024 con
 constexpr int kWarpSpan = 32 * kKeysPerLane;
 constexpr int kMaxWarpsPerUnit = 16;                    // T <= 16384
 
-// In-register transpose of a 32 x 32 bit matrix (row i = word a[i], column c = bit 31 - c):
-// five butterfly stages of masked swaps between words.
-__device__ __forceinline__ void transpose32(uint32_t (&a)[32])
+// Transpose of a 32 x 32 bit matrix held as one column of shared memory per lane (word i of the
+// lane = m[i * 32], row i of the matrix; column c = bit 31 - c): five butterfly stages of masked
+// swaps between words. Kept as loops on purpose: a selection warp runs this code once, so compact
+// code (few instruction-cache misses) matters more than instruction count.
+__device__ __forceinline__ void transpose32(uint32_t *m)
 {
-    uint32_t m = 0x0000FFFFu;
-#pragma unroll
+    uint32_t mask = 0x0000FFFFu;
+#pragma unroll 1
     for (int j = 16; j != 0; j >>= 1) {
-#pragma unroll
-        for (int k = 0; k < 32; ++k) {
-            if ((k & j) == 0) {
-                const uint32_t t = (a[k] ^ (a[k + j] >> j)) & m;
-                a[k] ^= t;
-                a[k + j] ^= t << j;
-            }
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+            const int k = ((i & ~(j - 1)) << 1) | (i & (j - 1));      // i-th index with bit j clear
+            const uint32_t lo = m[k * 32], hi = m[(k + j) * 32];
+            const uint32_t t = (lo ^ (hi >> j)) & mask;
+            m[k * 32] = lo ^ t;
+            m[(k + j) * 32] = hi ^ (t << j);
         }
-        m ^= m << (j >> 1);
+        mask ^= mask << (j >> 1);
     }
 }
 
@@ -54,7 +56,7 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32])
 // independent units, one per warp, and no block-wide barrier is ever needed. Lane l of warp w owns
 // positions 1024*w + 32*j + l (j = 0..31, its "rows").
 //  1. The lane's 32 keys (order-preserving uint32 images of the scores) are transposed into 32
-//     bit planes, so "how many of my still-undecided keys have bit b set" is one AND and one popc.
+//     bit planes (a shared-memory column per lane), so "how many of my still-undecided keys have bit b set" is one AND and one popc.
 //  2. Radix descent from the top bit for the C-th largest key: if at least `need` undecided keys of
 //     the unit have the bit set, those stay undecided and the others are out; otherwise they are all
 //     anchors (`greater`), `need` shrinks by their count and the others stay undecided. All keys
@@ -70,6 +72,7 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
               int32_t *__restrict__ anchor_pos, int32_t *__restrict__ bucket_len)
 {
     __shared__ uint32_t xa[2][kMaxWarpsPerUnit], xb[kMaxWarpsPerUnit];     // cross-warp exchange (G > 1)
+    extern __shared__ uint32_t planes_all[];                               // 32 x 32 words per warp
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int unit = (G == 1) ? blockIdx.x * 4 + warp : blockIdx.x;
     if (G == 1 && unit >= n_units) return;                 // whole warp leaves; no barriers in this variant
@@ -92,26 +95,29 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
         return t;
     };
 
-    // a[31 - j] = key of row j, so that after the transpose a[31 - b] is the plane of key bit b with
-    // row j at mask bit j
-    uint32_t a[32];
+    // pl[(31 - j) * 32] = key of row j, so that after the transpose pl[(31 - b) * 32] is the plane of
+    // key bit b with row j at mask bit j (one shared-memory column per lane: conflict-free)
+    uint32_t *pl = planes_all + warp * 1024 + lane;
     uint32_t undecided = 0u, greater = 0u;                 // row masks
     uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;               // range of the unprotected keys
+    {
+        float raw[kKeysPerLane];
 #pragma unroll
-    for (int j = 0; j < kKeysPerLane; ++j) {               // all loads first, so that they overlap
-        const int t = base + 32 * j + lane;
-        a[31 - j] = (t < T) ? __float_as_uint(__ldg(s + t)) : 0u;
-    }
-#pragma unroll
-    for (int j = 0; j < kKeysPerLane; ++j) {
-        const int t = base + 32 * j + lane;
-        uint32_t key = 0u;
-        if (t < T) {
-            key = sort_key(__uint_as_float(a[31 - j]));
-            if (is_prot(t)) greater |= 1u << j;
-            else { undecided |= 1u << j; kmin = min(kmin, key); kmax = max(kmax, key); }
+        for (int j = 0; j < kKeysPerLane; ++j) {           // all loads first, so that they overlap
+            const int t = base + 32 * j + lane;
+            raw[j] = (t < T) ? __ldg(s + t) : 0.f;
         }
-        a[31 - j] = key;
+#pragma unroll
+        for (int j = 0; j < kKeysPerLane; ++j) {
+            const int t = base + 32 * j + lane;
+            uint32_t key = 0u;
+            if (t < T) {
+                key = sort_key(raw[j]);
+                if (is_prot(t)) greater |= 1u << j;
+                else { undecided |= 1u << j; kmin = min(kmin, key); kmax = max(kmax, key); }
+            }
+            pl[(31 - j) * 32] = key;
+        }
     }
     kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
     kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
@@ -122,25 +128,24 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
         for (int w = 0; w < G; ++w) { kmin = min(kmin, xa[par][w]); kmax = max(kmax, xb[w]); }
         par ^= 1;
     }
-    transpose32(a);
+    transpose32(pl);
 
     uint32_t need = (uint32_t)(C - nprot);                // anchors still to find among the unprotected keys
     if (need == 0) {
         undecided = 0u;                                   // only the protected keys are anchors
     } else if (kmin != kmax) {                            // (kmin == kmax: every unprotected key is a tie)
         const int nbits = 32 - __clz(kmin ^ kmax);
-#pragma unroll
-        for (int b = 31; b >= 0; --b) {
-            if (b < nbits) {                              // uniform over the unit
-                const uint32_t ones = undecided & a[31 - b];
-                const uint32_t c1 = unit_sum(__popc(ones));
-                if (c1 >= need) {
-                    undecided = ones;
-                } else {
-                    need -= c1;
-                    greater |= ones;
-                    undecided &= ~a[31 - b];
-                }
+#pragma unroll 1
+        for (int b = nbits - 1; b >= 0; --b) {            // uniform over the unit
+            const uint32_t plane = pl[(31 - b) * 32];
+            const uint32_t ones = undecided & plane;
+            const uint32_t c1 = unit_sum(__popc(ones));
+            if (c1 >= need) {
+                undecided = ones;
+            } else {
+                need -= c1;
+                greater |= ones;
+                undecided &= ~plane;
             }
         }
     }
@@ -161,7 +166,7 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
 
     const uint32_t lt_mask = (1u << lane) - 1u;
     int32_t *ap0 = anchor_pos + (size_t)unit * replicate * C;
-#pragma unroll
+#pragma unroll 2
     for (int j = 0; j < kKeysPerLane; ++j) {
         const bool is_gt = (greater >> j) & 1u, is_eq = (undecided >> j) & 1u;
         const uint32_t bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
@@ -201,7 +206,12 @@ cudaError_t launch_select_t(const float *scores, int n_units, int T, int n_keep,
                             int32_t *anchor_pos, int32_t *bucket_len, cudaStream_t stream)
 {
     const unsigned grid = (G == 1) ? (unsigned)((n_units + 3) / 4) : (unsigned)n_units;
-    select_kernel<G><<<grid, G == 1 ? 128 : 32 * G, 0, stream>>>(scores, n_units, T, n_keep, protect_ends, replicate,
+    constexpr int smem = (G == 1 ? 4 : G) * 32 * 32 * (int)sizeof(uint32_t);      // bit planes: 4 KB per warp
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(select_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+    }
+    select_kernel<G><<<grid, G == 1 ? 128 : 32 * G, smem, stream>>>(scores, n_units, T, n_keep, protect_ends, replicate,
                                                                  anchor_pos, bucket_len);
     return cudaGetLastError();
 }
