@@ -109,7 +109,7 @@ int ec_importance_prefix(const void *Q_dev, const void *K_dev, float *scores_dev
  * the model's own forward pass, Algorithm 1 "Input"): only the column-sum pass runs, which
  * halves the contraction work.
  *   lse_dev   fp32 [N, H, T], natural log of sum_{n<=m} exp(scale*<q_m,k_n>), same `scale`  (in)
- * Other arguments, workspace size and limits as ec_importance; additionally N*H <= 65535.
+ * Other arguments, workspace size and limits as ec_importance.
  */
 int ec_importance_from_lse(const void *Q_dev, const void *K_dev, const float *lse_dev, float *scores_dev,
                            int N, int H, int T, int D, float scale,
@@ -172,7 +172,7 @@ int ec_select_merge(const void *K_dev, const void *V_dev, const float *scores_de
  *   share       how many consecutive units rank one common score vector (the mean of their
  *               scores): 1 = head-wise, H = layer-wise, layers*H = one selection per sequence
  *               ("identical" for all layers; problems n = b*layers + l must be layer-minor).
- *               N*H must be a multiple of share; N*H/share <= 65535 when share > 1.
+ *               N*H must be a multiple of share.
  *   compaction  EC_COMPACT_MERGE: bucket means (Eq. 3).  EC_COMPACT_EVICT: the kept rows are
  *               the anchors' own rows and all other rows are dropped.
  * Everything else as ec_select_merge, which is this call with share = 1 or H and

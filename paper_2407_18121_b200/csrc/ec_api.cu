@@ -94,7 +94,6 @@ int ec_importance_from_lse(const void *Q, const void *K, const float *lse, float
     if (!Q || !K || !scores || !lse) return EC_ERR_NULL;
     int st = check_shape(N, H, T, D);
     if (st != EC_OK) return st;
-    if ((long long)N * H > 65535) return EC_ERR_SHAPE;
     if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || !aligned(lse, 4)) return EC_ERR_ALIGN;
     if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
@@ -139,7 +138,6 @@ int ec_select_compact(const void *K, const void *V, const float *scores, int N, 
     if (st != EC_OK) return st;
     if (n_keep < 1 || n_keep > T || cap < n_keep) return EC_ERR_ARG;
     if (share < 1 || ((long long)N * H) % share != 0) return EC_ERR_ARG;
-    if (share > 1 && (long long)N * H / share > 65535) return EC_ERR_SHAPE;
     if (compaction != EC_COMPACT_MERGE && compaction != EC_COMPACT_EVICT) return EC_ERR_ARG;
     if ((long long)N * H * cap >= (1LL << 31)) return EC_ERR_SHAPE;
     if (!aligned(K, 16) || !aligned(V, 16) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(scores, 4) ||

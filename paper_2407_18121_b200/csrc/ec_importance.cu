@@ -527,8 +527,8 @@ bool make_map(CUtensorMap *map, const void *ptr, int units, int T, int D)
 // A caller-provided natural-log normaliser [units, T] -> the padded log2-domain layout pass 2 reads.
 __global__ void lse_import_kernel(const float *__restrict__ lse_nat, float *__restrict__ lse2, int T, int Tpad)
 {
-    const int unit = blockIdx.y;
-    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    const int unit = blockIdx.x;
+    const int m = blockIdx.y * blockDim.x + threadIdx.x;
     if (m >= Tpad) return;
     lse2[(size_t)unit * Tpad + m] = (m < T) ? lse_nat[(size_t)unit * T + m] * kLog2e : INFINITY;
 }
@@ -611,8 +611,7 @@ cudaError_t launch_importance(const void *Q, const void *K, float *scores, float
     CUtensorMap mq, mk;
     if (!make_map(&mq, Q, units, Tq, D) || !make_map(&mk, K, units, Tq + P, D)) return cudaErrorInvalidValue;
     if (lse_in) {
-        if (units > 65535) return cudaErrorInvalidConfiguration;
-        dim3 g((geo.ntq * kTileRows + 255) / 256, units);
+        dim3 g(units, (geo.ntq * kTileRows + 255) / 256);
         lse_import_kernel<<<g, 256, 0, stream>>>(lse_in, lse2, Tq, geo.ntq * kTileRows);
     }
     const float c = scale * kLog2e;

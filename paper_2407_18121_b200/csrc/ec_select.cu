@@ -18,8 +18,8 @@ __device__ __forceinline__ uint32_t sort_key(float x)
 // layer and head of a sequence). scores [G*share, T] -> mean [G, T].
 __global__ void group_mean_kernel(const float *__restrict__ scores, float *__restrict__ mean, int share, int T)
 {
-    const size_t grp = blockIdx.y;
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t grp = blockIdx.x;
+    const int t = blockIdx.y * blockDim.x + threadIdx.x;
     if (t >= T) return;
     const float *s = scores + grp * share * T + t;
     float acc = 0.f;
@@ -225,8 +225,7 @@ cudaError_t launch_select(const float *scores, int units, int T, int n_keep, int
     int n = units, rep = 1;
     if (share > 1) {
         const int groups = units / share;
-        if (groups > 65535) return cudaErrorInvalidConfiguration;
-        dim3 g((T + 255) / 256, groups);
+        dim3 g(groups, (T + 255) / 256);
         group_mean_kernel<<<g, 256, 0, stream>>>(scores, mean_ws, share, T);
         src = mean_ws;
         n = groups;

@@ -665,3 +665,27 @@ def test_whole_pass_can_be_captured_in_a_cuda_graph_and_replayed():
         assert torch.equal(out_graph, out_eager)
         assert torch.equal(sess.Kc, Kc_ref) and torch.equal(sess.anchor_pos, anchors_ref)
     assert ec.ec_device_status(sess.ws_imp) == ec.EC_OK
+
+
+def test_ratio_policy_through_the_overlapped_native_loop():
+    """Growing cache + native loop with one CTA per unit: the row the previous step appended (or
+    overwrote) is the one read late. Must equal the one-step calls."""
+    rng = np.random.default_rng(31)
+    N, H, D, C, d, S, T, ratio = 20, 32, 128, 41, 9, 30, 100, 0.41
+    cap = C + S
+    K0, V0 = (dev_bf16(rand_bits(rng, (N, H, cap, D))) for _ in range(2))
+    q, k, v = (dev_bf16(rand_bits(rng, (S, N, H, D))) for _ in range(3))
+    Ka, Va, Kb_, Vb_ = K0.clone(), V0.clone(), K0.clone(), V0.clone()
+    ca = ec.ec_cache_init_ratio(Ka, Va, C, d, ratio, T)
+    cb = ec.ec_cache_init_ratio(Kb_, Vb_, C, d, ratio, T)
+    ws = scratch(ec.ec_decode_workspace(ca))
+    out_a = torch.empty((S, N, H, D), dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty_like(out_a)
+    slots_a = [ec.ec_decode_step(q[s], k[s], v[s], ca, 0.09, out_a[s], ws)[0] for s in range(S)]
+    slots_b = ec.ec_decode_steps(q, k, v, cb, 0.09, out_b, ws, want_slots=True)
+    torch.cuda.synchronize()
+    assert slots_a == slots_b and -1 in slots_a and any(x >= 0 for x in slots_a)    # grew and evicted
+    assert (ca.len, ca.n_tot, ca.recent_head) == (cb.len, cb.n_tot, cb.recent_head)
+    assert torch.equal(Ka[:, :, :ca.len], Kb_[:, :, :cb.len]) and torch.equal(Va[:, :, :ca.len], Vb_[:, :, :cb.len])
+    a, b = host_f64(out_a), host_f64(out_b)
+    assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(a) + 1e-6).all()
