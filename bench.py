@@ -382,7 +382,7 @@ def run_ours(args, w: wl.Workload):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 storage, fp32 arithmetic", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32", "storage_dtype": "bf16", "data": "synthetic",
         "config": workload_config(w),
         "stages_ms": {"importance": imp_ms, "select_merge": mrg_ms, "decode_loop": dec_ms,
                       "decode_per_token_us": dec_ms * 1e3 / S, "whole_pass_cuda_graph_replay": graph_ms},
