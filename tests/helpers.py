@@ -4,7 +4,7 @@ import torch
 
 from paper_2407_18121_b200 import workloads as wl
 
-# Tolerances (stated by the benchmark spec for this path):
+# Tolerances of the parity checks:
 #   fp32 results (importance scores, lse): relative 1e-3
 #   bf16 results (merged K/V rows, decode outputs): |gpu - oracle| <= 2e-2 + 2^-8 * |oracle|
 #   (the relative term is bf16's own half-ulp bound, which exceeds 2e-2 once |x| >= 8)
