@@ -11,10 +11,16 @@
  *   ec_decode_step   single-query attention over the compacted cache plus the new token,
  *                    followed by fixed-point elimination (in-place slot reuse)
  *
+ * plus variants of each (importance on top of cached rows or from a known log-sum-exp,
+ * shared populations and eviction-only compaction, a native multi-step decode loop, the
+ * retention-ratio policy, host-resident tensors, a decode step with built-in scratch).
+ *
  * Conventions shared by every call
  *  - Pointers named "dev" are CUDA device pointers of the current device; "host" pointers
- *    are ordinary host memory. The caller owns every buffer. The library allocates no
- *    device memory and keeps no state between calls.
+ *    are ordinary host memory. The caller owns every buffer. No call allocates device
+ *    memory, and no call depends on an earlier one except through the buffers and the
+ *    ec_cache struct the caller passes (the library only caches a driver entry point and,
+ *    for ec_decode_step_noalloc, the address of its built-in scratch).
  *  - bf16 tensors are passed as `const void*` to 2-byte elements, row-major, innermost
  *    dimension contiguous, base address 16-byte aligned. D (head_dim) is 64 or 128.
  *  - N counts independent problems (batch x layers folded), H heads per problem. A "unit"
