@@ -38,7 +38,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one decode_kernel launch from the ncu capture summarised in
 # profiles/decode_kernel_llava7b_b1_ncu.md, keyed by workload; valid only for the kernel source it was
 # taken on (sha1 prefix of csrc/ec_decode.cu), otherwise reported as null.
-DECODE_TRAFFIC = {"source_sha1": "f185b30eaa7e", "llava7b_b1": 172.15e6}
+DECODE_TRAFFIC = {"source_sha1": "ac8fbbb5c83f", "llava7b_b1": 172.17e6}
 
 
 def decode_traffic(workload: str):

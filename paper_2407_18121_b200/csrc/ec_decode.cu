@@ -34,6 +34,16 @@ __device__ __forceinline__ uint4 ld_row(const uint4 *p)
     return v;
 }
 
+// Same load served from L2: used for the rows read after waiting for the previous step, so that a
+// line which an earlier read of a neighbouring row may have left in L1 cannot be served stale.
+__device__ __forceinline__ uint4 ld_row_l2(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -67,7 +77,8 @@ struct GroupState {
 
 // One block of up to 8 consecutive cache rows starting at `row`. GUARD: rows >= row_end are
 // skipped (their loads are clamped to the last valid row and their score is -inf).
-template <int LPR, bool GUARD>
+// FRESH: the block is read after the wait for the previous step and must not come from L1.
+template <int LPR, bool GUARD, bool FRESH = false>
 __device__ __forceinline__ void process_block(GroupState &st, const float2 (&q2)[4], const uint4 *Kl, const uint4 *Vl,
                                               int row, int row_end, int l, unsigned gmask)
 {
@@ -75,12 +86,12 @@ __device__ __forceinline__ void process_block(GroupState &st, const float2 (&q2)
 #pragma unroll
     for (int r = 0; r < kBlk; ++r) {
         const int j = GUARD ? min(row + r, row_end - 1) : row + r;
-        rk[r] = ld_row(Kl + (size_t)j * LPR);
+        rk[r] = FRESH ? ld_row_l2(Kl + (size_t)j * LPR) : ld_row(Kl + (size_t)j * LPR);
     }
 #pragma unroll
     for (int r = 0; r < kBlk; ++r) {
         const int j = GUARD ? min(row + r, row_end - 1) : row + r;
-        rv[r] = ld_row(Vl + (size_t)j * LPR);
+        rv[r] = FRESH ? ld_row_l2(Vl + (size_t)j * LPR) : ld_row(Vl + (size_t)j * LPR);
     }
     float s[kBlk];
 #pragma unroll
@@ -191,8 +202,8 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
         grid_dependency_wait();
         grid_launch_dependents();
         if (bd >= 0 && (bd % G) == g) {
-            if (bd < nfull) process_block<LPR, false>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
-            else            process_block<LPR, true>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
+            if (bd < nfull) process_block<LPR, false, true>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
+            else            process_block<LPR, true, true>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
         }
     }
 
