@@ -689,3 +689,39 @@ def test_ratio_policy_through_the_overlapped_native_loop():
     assert torch.equal(Ka[:, :, :ca.len], Kb_[:, :, :cb.len]) and torch.equal(Va[:, :, :ca.len], Vb_[:, :, :cb.len])
     a, b = host_f64(out_a), host_f64(out_b)
     assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(a) + 1e-6).all()
+
+
+# ---------------------------------------------------------------- seeded random shapes
+
+def test_random_shapes_select_merge_and_decode():
+    """Forty seeded shapes off the beaten path (prompt lengths around warp / tile / slice borders,
+    keep counts from 1 to T, both head sizes, shared populations, long offsets)."""
+    rng = np.random.default_rng(20240718)
+    for case in range(40):
+        D = int(rng.choice([64, 128]))
+        H = int(rng.integers(1, 5))
+        N = int(rng.integers(1, 4))
+        T = int(rng.choice([1, 2, 3, 31, 32, 33, 63, 255, 256, 257, 511, 513, 1023, 1024, 1025, 1500, 2049]))
+        n_keep = int(rng.integers(1, T + 1))
+        protect = bool(rng.integers(0, 2))
+        share = int(rng.choice([1, H]))
+        Kb, Vb = rand_bits(rng, (N, H, T, D)), rand_bits(rng, (N, H, T, D))
+        levels = int(rng.choice([3, 50, 100000]))                      # few levels -> many exact ties
+        s32 = (rng.integers(1, levels + 1, size=(N, H, T)) / levels).astype(np.float32)
+        rank = np.repeat(orc.group_mean(s32.astype(np.float64).reshape(N * H, T), share), share, 0).reshape(N, H, T)
+        want = orc.select(rank, n_keep, protect)
+        Kc, Vc, anchors = gpu_select_compact(Kb, Vb, s32, n_keep, share, protect, ec.EC_COMPACT_MERGE)
+        exact, total = check_anchor_sets(anchors, want, rank, n_keep, protect)
+        if share == 1:
+            assert exact == total, (case, N, H, T, D, n_keep, protect)
+        lo, hi = orc.buckets(anchors_to_merge_on(anchors, want), T)
+        assert_bf16_close(Kc, orc.merge(Kb, lo, hi), f"merged K, case {case}")
+        assert_bf16_close(Vc, orc.merge(Vb, lo, hi), f"merged V, case {case}")
+    for case in range(12):
+        D = int(rng.choice([64, 128]))
+        N, H = int(rng.integers(1, 30)), int(rng.integers(1, 33))
+        C = int(rng.integers(2, 150))
+        offset = int(rng.integers(1, C))
+        len0 = int(rng.integers(0, C + 1))
+        run_decode_case(N, H, D, C, C + int(rng.integers(0, 5)), len0, offset, int(rng.integers(1, 12)),
+                        float(rng.uniform(0.05, 0.3)), seed=1000 + case)
