@@ -142,42 +142,50 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32])
     for (int i = 0; i < 32; ++i) asm volatile("" : "+r"(r[i]));
 }
 
-// 2^x on the FMA pipe (Cody-Waite split + degree-4 polynomial, relative error < 6e-6) for
-// x <= ~0. With EC_IMP_POLY_EVERY = n > 0, one element in n goes this way to take load off the
-// special-function unit (one ex2 per score element is the busiest pipe of these kernels).
-// Off by default: measured on B200 it does not pay (n = 4: -1..+1%, n = 3: -5%), because with
-// two CTAs per SM the softmax warps wait on TMEM loads and barriers more than on the ex2 pipe.
-#ifndef EC_IMP_POLY_EVERY
-#define EC_IMP_POLY_EVERY 0          // 0 = never
+// One ex2 per score element makes the special-function unit the busiest pipe of these kernels
+// (16 results per clock per SM). One element pair in EC_IMP_POLY_PAIR_EVERY is therefore evaluated
+// on the FMA pipe instead, with packed fp32 pair instructions: Cody-Waite split and a degree-4
+// polynomial, relative error < 6e-6, inputs clamped at -125 (so a masked -inf gives 2^-125, far
+// below one ulp of any sum it joins). Measured on B200: +3% at T = 640, +6-8% at T >= 2048 with
+// one pair in four; one in three or two is slower again. 0 turns it off.
+#ifndef EC_IMP_POLY_PAIR_EVERY
+#define EC_IMP_POLY_PAIR_EVERY 4
 #endif
-__device__ __forceinline__ float poly_exp2(float x)
+__device__ __forceinline__ float2 poly_exp2_pair(float2 x)
 {
-    x = fmaxf(x, -125.f);                               // below this the result is ~0 anyway
-    const float t = x + 12582912.f;                     // 1.5 * 2^23: the low mantissa bits now hold round(x)
-    const float f = x - (t - 12582912.f);               // fractional part in [-0.5, 0.5]
-    float p = fmaf(f, 0.00935919489711523f, 0.05588679388165474f);
-    p = fmaf(p, f, 0.2402936965227127f);
-    p = fmaf(p, f, 0.6931265592575073f);
-    p = fmaf(p, f, 0.9999980926513672f);
-    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));   // scale by 2^round(x)
+    const float2 magic = make_float2(12582912.f, 12582912.f);       // 1.5 * 2^23: low mantissa bits = round(x)
+    const float2 nmagic = make_float2(-12582912.f, -12582912.f), neg1 = make_float2(-1.f, -1.f);
+    x.x = fmaxf(x.x, -125.f);
+    x.y = fmaxf(x.y, -125.f);
+    const float2 t = __fadd2_rn(x, magic);
+    const float2 f = __ffma2_rn(__fadd2_rn(t, nmagic), neg1, x);    // fractional part in [-0.5, 0.5]
+    float2 p = __ffma2_rn(f, make_float2(0.00935919489711523f, 0.00935919489711523f),
+                          make_float2(0.05588679388165474f, 0.05588679388165474f));
+    p = __ffma2_rn(p, f, make_float2(0.2402936965227127f, 0.2402936965227127f));
+    p = __ffma2_rn(p, f, make_float2(0.6931265592575073f, 0.6931265592575073f));
+    p = __ffma2_rn(p, f, make_float2(0.9999980926513672f, 0.9999980926513672f));
+    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),   // scale by 2^round(x)
+                       __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
 }
 
-template <int I>
-__device__ __forceinline__ float exp2_mixed(float x)
+// 2^a for a pair; `pair_index` is a compile-time constant after unrolling.
+__device__ __forceinline__ float2 exp2_pair(float2 a, int pair_index)
 {
-    constexpr int every = EC_IMP_POLY_EVERY > 0 ? EC_IMP_POLY_EVERY : 1;
-    if (EC_IMP_POLY_EVERY > 0 && (I % every) == every - 1) return poly_exp2(x);
-    return fast_exp2(x);
+    constexpr int every = EC_IMP_POLY_PAIR_EVERY > 0 ? EC_IMP_POLY_PAIR_EVERY : 1;
+    if (EC_IMP_POLY_PAIR_EVERY > 0 && pair_index % every == 0) return poly_exp2_pair(a);
+    return make_float2(fast_exp2(a.x), fast_exp2(a.y));
 }
 
-// part[i & 3] += 2^(v[i]*c - m) over the 32 values of a chunk, unrolled at compile time so that
-// the choice between ex2 and the polynomial is static per element.
-template <int I>
-__device__ __forceinline__ void sum_exp2(const float (&v)[32], float c, float m, float (&part)[4])
+// part[k] += 2^(v*c - m) over the 32 values of a chunk, two elements per instruction: the
+// scale-and-shift and the accumulation are packed fp32 pairs, only the ex2 itself is scalar.
+// Element i lands in chain i & 3, as a scalar loop over four chains would put it.
+__device__ __forceinline__ void sum_exp2(const float (&v)[32], float c, float m, float2 (&part)[2])
 {
-    if constexpr (I < 32) {
-        part[I & 3] += exp2_mixed<I>(fmaf(v[I], c, -m));
-        sum_exp2<I + 1>(v, c, m, part);
+    const float2 c2 = make_float2(c, c), nm = make_float2(-m, -m);
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const float2 a = __ffma2_rn(make_float2(v[i], v[i + 1]), c2, nm);
+        part[(i >> 1) & 1] = __fadd2_rn(part[(i >> 1) & 1], exp2_pair(a, i >> 1));
     }
 }
 
@@ -373,7 +381,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (!item_of(sidx, sub, unit, st, first, count)) break;
                 const size_t lse_row = (size_t)unit * geo.ntq * kTileRows;
                 float mrun = -INFINITY, Z = 0.f;                      // pass 1 running max / sum (log2 domain)
-                float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f; // pass 2 column sum
+                float2 accA = make_float2(0.f, 0.f), accB = accA;     // pass 2 column sum, four chains
                 float lse_ahead = 0.f;
                 if (PASS2 && half == 0) lse_ahead = lse2[lse_row + (size_t)first * kTileRows + r];
                 for (int t = 0; t < count; ++t, ++tg) {
@@ -390,7 +398,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         // (bounded) for the 128 entries; the buffer is reused two tiles later, after the
                         // next tile's rendezvous
                         if (half == 0) {
-                            lse_s[b * kTileRows + r] = lse_ahead;
+                            lse_s[b * kTileRows + r] = -lse_ahead;    // staged negated: exponent = v*c + (-lse)
                             mbar_arrive(bar_lse(b));
                             if (t + 1 < count)
                                 lse_ahead = lse2[lse_row + (size_t)stream_tile(first, t + 1) * kTileRows + r];
@@ -417,28 +425,30 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
                             const float mnew = fmaxf(mrun, cm * c);
                             if (mnew != -INFINITY) {
-                                float part[4] = {0.f, 0.f, 0.f, 0.f};
-                                sum_exp2<0>(v, c, mnew, part);
-                                Z = Z * fast_exp2(mrun - mnew) + ((part[0] + part[1]) + (part[2] + part[3]));
+                                float2 part[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                                sum_exp2(v, c, mnew, part);
+                                Z = Z * fast_exp2(mrun - mnew) + ((part[0].x + part[0].y) + (part[1].x + part[1].y));
                                 mrun = mnew;
                             }
                         } else {
                             const float4 *ls = reinterpret_cast<const float4 *>(lse_s + b * kTileRows + ch * 32);
                             const int lim = r - off - ch * 32;                // columns i >= lim are visible
+                            const float2 c2 = make_float2(c, c);
 #pragma unroll
                             for (int i4 = 0; i4 < 8; ++i4) {
-                                const float4 l4 = ls[i4];
-                                float p0 = exp2_mixed<0>(fmaf(v[i4 * 4 + 0], c, -l4.x));
-                                float p1 = exp2_mixed<1>(fmaf(v[i4 * 4 + 1], c, -l4.y));
-                                float p2 = exp2_mixed<2>(fmaf(v[i4 * 4 + 2], c, -l4.z));
-                                float p3 = exp2_mixed<3>(fmaf(v[i4 * 4 + 3], c, -l4.w));
+                                const float4 nl = ls[i4];                     // -lse of four query rows
+                                const float2 a01 = __ffma2_rn(make_float2(v[i4 * 4 + 0], v[i4 * 4 + 1]), c2, make_float2(nl.x, nl.y));
+                                const float2 a23 = __ffma2_rn(make_float2(v[i4 * 4 + 2], v[i4 * 4 + 3]), c2, make_float2(nl.z, nl.w));
+                                const float2 e01 = exp2_pair(a01, i4 * 2), e23 = exp2_pair(a23, i4 * 2 + 1);
+                                float p0 = e01.x, p1 = e01.y, p2 = e23.x, p3 = e23.y;
                                 if (masked) {
                                     if (i4 * 4 + 0 < lim) p0 = 0.f;
                                     if (i4 * 4 + 1 < lim) p1 = 0.f;
                                     if (i4 * 4 + 2 < lim) p2 = 0.f;
                                     if (i4 * 4 + 3 < lim) p3 = 0.f;
                                 }
-                                acc0 += p0; acc1 += p1; acc2 += p2; acc3 += p3;
+                                accA = __fadd2_rn(accA, make_float2(p0, p1));
+                                accB = __fadd2_rn(accB, make_float2(p2, p3));
                             }
                         }
                     };
@@ -462,7 +472,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const uint32_t iph = it & 1u;
                 if (half == 1) {
                     if (!mbar_wait(bar_comb_empty, iph ^ 1u, abort_flag, status)) { alive = false; break; }
-                    comb_s[r] = PASS2 ? make_float2((acc0 + acc1) + (acc2 + acc3), 0.f) : make_float2(mrun, Z);
+                    comb_s[r] = PASS2 ? make_float2((accA.x + accA.y) + (accB.x + accB.y), 0.f) : make_float2(mrun, Z);
                     mbar_arrive(bar_comb_full);
                 } else {
                     if (!mbar_wait(bar_comb_full, iph, abort_flag, status)) { alive = false; break; }
@@ -476,7 +486,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         lse2[lse_row + row] = l2;
                         if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
                     } else if (row < Tk) {
-                        scores[(size_t)unit * Tk + row] = ((acc0 + acc1) + (acc2 + acc3)) + o.x;
+                        scores[(size_t)unit * Tk + row] = ((accA.x + accA.y) + (accB.x + accB.y)) + o.x;
                     }
                 }
                 ++it;
