@@ -19,6 +19,7 @@
 #include "ec_common.cuh"
 
 #include <cuda.h>
+#include <type_traits>
 
 namespace ec {
 
@@ -409,12 +410,13 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     tc_fence_after();
 
                     // `ch` = index of the 32-column chunk inside the 128-column tile
-                    auto chunk = [&](uint32_t (&raw)[32], int ch) {
+                    auto chunk = [&](uint32_t (&raw)[32], int ch, auto mask_tag) {
+                        constexpr bool MASKED = decltype(mask_tag)::value;
                         float v[32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]);
                         if (!PASS2) {
-                            if (masked) {
+                            if constexpr (MASKED) {
                                 const int lim = r + off - ch * 32;            // columns i <= lim are visible
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) if (i > lim) v[i] = -INFINITY;
@@ -441,7 +443,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                 const float2 a23 = __ffma2_rn(make_float2(v[i4 * 4 + 2], v[i4 * 4 + 3]), c2, make_float2(nl.z, nl.w));
                                 const float2 e01 = exp2_pair(a01, i4 * 2), e23 = exp2_pair(a23, i4 * 2 + 1);
                                 float p0 = e01.x, p1 = e01.y, p2 = e23.x, p3 = e23.y;
-                                if (masked) {
+                                if constexpr (MASKED) {
                                     if (i4 * 4 + 0 < lim) p0 = 0.f;
                                     if (i4 * 4 + 1 < lim) p1 = 0.f;
                                     if (i4 * 4 + 2 < lim) p2 = 0.f;
@@ -453,18 +455,23 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         }
                     };
 
-                    // this thread's 64 columns: the second 32 are in flight while the first are processed
-                    const uint32_t col0 = lane_addr + b * kTileRows;
-                    uint32_t ra[32], rb[32];
-                    tmem_ld32_async(col0, ra);
-                    tmem_ld_wait(ra);
-                    tmem_ld32_async(col0 + 32, rb);
-                    chunk(ra, half * 2);
-                    tmem_ld_wait(rb);
-                    tc_fence_before();                   // all TMEM reads of this tile are done:
-                    __syncwarp();                        // hand the accumulator back before the last chunk's math
-                    if (lane == 0) mbar_arrive(bar_acc_empty(b));
-                    chunk(rb, half * 2 + 1);
+                    // this thread's 64 columns: the second 32 are in flight while the first are processed.
+                    // Only tiles the diagonal crosses pay for the mask: they run a separate instance.
+                    auto tile_body = [&](auto mask_tag) {
+                        const uint32_t col0 = lane_addr + b * kTileRows;
+                        uint32_t ra[32], rb[32];
+                        tmem_ld32_async(col0, ra);
+                        tmem_ld_wait(ra);
+                        tmem_ld32_async(col0 + 32, rb);
+                        chunk(ra, half * 2, mask_tag);
+                        tmem_ld_wait(rb);
+                        tc_fence_before();                   // all TMEM reads of this tile are done:
+                        __syncwarp();                        // hand the accumulator back before the last chunk's math
+                        if (lane == 0) mbar_arrive(bar_acc_empty(b));
+                        chunk(rb, half * 2 + 1, mask_tag);
+                    };
+                    if (masked) tile_body(std::true_type{});
+                    else tile_body(std::false_type{});
                 }
                 if (!alive) break;
 
