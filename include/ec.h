@@ -313,6 +313,26 @@ int ec_decode_steps_host(const void *q_host, const void *k_host, const void *v_h
                          ec_cache *c, float scale, void *ws_dev, size_t ws_bytes,
                          void *stream, void *upload_stream, void *download_stream);
 
+/* ---------------------------------------------------------------- history for a new instruction */
+
+/*
+ * The key/value history a further instruction is encoded against (Sec. 3.1: the instruction
+ * stage takes in the chat history): the cache's rows in queue order, oldest first, followed
+ * by the Tq rows of the new tokens. The result feeds ec_importance_prefix (P = c->len) and
+ * ec_select_merge / ec_select_compact over T = c->len + Tq rows.
+ *   c                      fixed-budget cache (EC_POLICY_FIXED; the retention-ratio policy does
+ *                          not keep the queue order of old rows and returns EC_ERR_ARG);
+ *                          read only, c->len >= 1
+ *   K_new_dev, V_new_dev   device bf16 [N, H, Tq, D], 16-byte aligned, Tq >= 1
+ *   K_all_dev, V_all_dev   device bf16 [N, H, c->len + Tq, D], written; must not overlap
+ *                          the cache or the new rows
+ * Row j < len of a unit comes from physical slot j while j < budget - offset or the cache is
+ * not yet full, else from the ring: slot (budget - offset) + (ring_head + j - (budget - offset))
+ * mod offset. Rows are copied bit for bit. Asynchronous on `stream`.
+ */
+int ec_cache_concat(const ec_cache *c, const void *K_new_dev, const void *V_new_dev, int Tq,
+                    void *K_all_dev, void *V_all_dev, void *stream);
+
 /* ---------------------------------------------------------------- no-allocation decode */
 
 /*

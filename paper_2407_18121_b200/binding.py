@@ -16,7 +16,8 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libec.so")
 
-EC_OK = 0
+EC_OK, EC_ERR_NULL, EC_ERR_SHAPE, EC_ERR_ALIGN, EC_ERR_ARG = 0, 1, 2, 3, 4
+EC_ERR_WORKSPACE, EC_ERR_CUDA, EC_ERR_TIMEOUT, EC_ERR_TOO_LARGE = 5, 6, 7, 8
 EC_PER_HEAD = 0
 EC_LAYER_SHARED = 1
 
@@ -24,7 +25,7 @@ EXPORTS = (
     "ec_status_string", "ec_keep_count",
     "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_from_lse", "ec_device_status", "ec_selftest_wait_timeout",
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
-    "ec_cache_init", "ec_cache_init_ratio", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
+    "ec_cache_init", "ec_cache_init_ratio", "ec_cache_concat", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc", "ec_compress_host", "ec_decode_steps_host",
 )
 
@@ -87,6 +88,8 @@ def lib() -> C.CDLL:
     L.ec_cache_init_ratio.restype = i
     L.ec_cache_init_ratio.argtypes = [C.POINTER(ec_cache), vp, vp, i, i, i, i, i, i, C.c_double, C.c_int64,
                                       C.POINTER(C.c_int)]
+    L.ec_cache_concat.restype = i
+    L.ec_cache_concat.argtypes = [C.POINTER(ec_cache), vp, vp, i, vp, vp, vp]
     L.ec_decode_workspace.restype = sz
     L.ec_decode_workspace.argtypes = [C.POINTER(ec_cache)]
     L.ec_decode_step.restype = i
@@ -260,6 +263,18 @@ def ec_decode_steps(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, c
                                slots, _ptr(ws), ws.numel() * ws.element_size(), _stream())
     _check(st, "ec_decode_steps")
     return list(slots) if want_slots else None
+
+
+def ec_cache_concat(cache: ec_cache, K_new: torch.Tensor, V_new: torch.Tensor, K_all: torch.Tensor,
+                    V_all: torch.Tensor) -> None:
+    """K_all, V_all [N,H,len+Tq,D] <- the cache's rows in queue order, then K_new, V_new [N,H,Tq,D]."""
+    Tq = K_new.shape[2]
+    if tuple(K_all.shape) != (cache.N, cache.H, cache.len + Tq, cache.D) or K_all.shape != V_all.shape:
+        raise ValueError("K_all, V_all must be [N, H, len + Tq, D]")
+    if tuple(K_new.shape) != (cache.N, cache.H, Tq, cache.D) or K_new.shape != V_new.shape:
+        raise ValueError("K_new, V_new must be [N, H, Tq, D]")
+    st = lib().ec_cache_concat(C.byref(cache), _ptr(K_new), _ptr(V_new), Tq, _ptr(K_all), _ptr(V_all), _stream())
+    _check(st, "ec_cache_concat")
 
 
 def ec_decode_noalloc_capacity() -> int:

@@ -190,6 +190,24 @@ int ec_cache_init(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, int cap,
     return EC_OK;
 }
 
+int ec_cache_concat(const ec_cache *c, const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
+                    void *stream)
+{
+    if (!c || !K_new || !V_new || !K_all || !V_all || !c->Kc || !c->Vc) return EC_ERR_NULL;
+    if (c->policy != EC_POLICY_FIXED) return EC_ERR_ARG;
+    if (c->N < 1 || c->H < 1 || (c->D != 64 && c->D != 128)) return EC_ERR_SHAPE;
+    if (Tq < 1 || c->len < 1 || c->len > c->budget || c->budget > c->cap) return EC_ERR_ARG;
+    if (c->offset < 1 || c->offset > c->budget - 1 || c->ring_head < 0 || c->ring_head >= c->offset) return EC_ERR_ARG;
+    const long long units = (long long)c->N * c->H;
+    if (units * ((long long)c->len + Tq) >= (1LL << 31)) return EC_ERR_SHAPE;
+    if (!aligned(K_new, 16) || !aligned(V_new, 16) || !aligned(K_all, 16) || !aligned(V_all, 16)) return EC_ERR_ALIGN;
+    const bool full = c->len == c->budget;               // the ring exists once the cache has reached its budget
+    cudaError_t e = ec::launch_concat(c->Kc, c->Vc, (int)units, c->cap, c->D, c->len, full ? c->budget - c->offset : c->len,
+                                      full ? c->offset : 0, full ? c->ring_head : 0, K_new, V_new, Tq, K_all, V_all,
+                                      (cudaStream_t)stream);
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
 int ec_cache_init_ratio(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, int cap, int len, int offset,
                         double keep_ratio, int64_t n_tot, int *recent_slots)
 {

@@ -65,6 +65,12 @@ cudaError_t launch_select(const float *scores, int units, int T, int n_keep, int
                           int32_t *anchor_pos, int32_t *bucket_len, float *mean_ws, cudaStream_t stream);
 cudaError_t launch_gather(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
                           int n_keep, void *Kc, void *Vc, int cap, cudaStream_t stream);
+
+// K_all/V_all [units, P + Tq, D] <- cache rows in queue order (slot j below `base`, ring slots
+// base + (ring_head + j - base) % ring after it; ring = 0 means no ring yet) followed by the new rows.
+cudaError_t launch_concat(const void *Kc, const void *Vc, int units, int cap, int D, int P, int base, int ring,
+                          int ring_head, const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
+                          cudaStream_t stream);
 cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
                          int n_keep, void *Kc, void *Vc, int cap, cudaStream_t stream);
 

@@ -146,6 +146,35 @@ gather_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const in
     *dst = ldg_stream(src);
 }
 
+// History for a further instruction: output row j of a unit is cache row j in queue order for
+// j < P, new row j - P after it. One lane group per output row, K on its first half, V on the second.
+template <int LPR>
+__global__ void __launch_bounds__(kMergeThreads)
+concat_kernel(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, int cap, int P, int base, int ring,
+              int ring_head, const uint4 *__restrict__ K_new, const uint4 *__restrict__ V_new, int Tq, int chunks,
+              uint4 *__restrict__ K_all, uint4 *__restrict__ V_all)
+{
+    constexpr int GL = 2 * LPR;
+    constexpr int G = kMergeThreads / GL;
+    const int unit = blockIdx.x / chunks;
+    const int chunk = blockIdx.x - unit * chunks;
+    const int g = threadIdx.x / GL, gl = threadIdx.x - g * GL;
+    const bool is_v = gl >= LPR;
+    const int l = is_v ? gl - LPR : gl;
+    const int j = chunk * G + g;
+    const int T = P + Tq;
+    if (j >= T) return;
+    const uint4 *src;
+    if (j < P) {
+        const int slot = (j < base || ring == 0) ? j : base + (ring_head + (j - base)) % ring;
+        src = (is_v ? Vc : Kc) + ((size_t)unit * cap + slot) * LPR + l;
+    } else {
+        src = (is_v ? V_new : K_new) + ((size_t)unit * Tq + (j - P)) * LPR + l;
+    }
+    uint4 *dst = (is_v ? V_all : K_all) + ((size_t)unit * T + j) * LPR + l;
+    *dst = ldg_stream(src);
+}
+
 template <int LPR>
 cudaError_t launch_merge_t(const void *K, const void *V, const int32_t *anchor_pos, unsigned grid, int T, int n_keep,
                            int slices, void *Kc, void *Vc, int cap, cudaStream_t stream)
@@ -190,6 +219,19 @@ cudaError_t launch_gather_t(const void *K, const void *V, const int32_t *anchor_
                               (uint4 *)Kc, (uint4 *)Vc, cap);
 }
 
+template <int LPR>
+cudaError_t launch_concat_t(const void *Kc, const void *Vc, int units, int cap, int P, int base, int ring, int ring_head,
+                            const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all, cudaStream_t stream)
+{
+    constexpr int G = kMergeThreads / (2 * LPR);
+    const int chunks = (P + Tq + G - 1) / G;
+    if ((long long)units * chunks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    concat_kernel<LPR><<<(unsigned)(units * chunks), kMergeThreads, 0, stream>>>(
+        (const uint4 *)Kc, (const uint4 *)Vc, cap, P, base, ring, ring_head, (const uint4 *)K_new, (const uint4 *)V_new, Tq,
+        chunks, (uint4 *)K_all, (uint4 *)V_all);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
@@ -207,6 +249,15 @@ cudaError_t launch_gather(const void *K, const void *V, const int32_t *anchor_po
 {
     if (D == 128) return launch_gather_t<16>(K, V, anchor_pos, units, T, n_keep, Kc, Vc, cap, stream);
     return launch_gather_t<8>(K, V, anchor_pos, units, T, n_keep, Kc, Vc, cap, stream);
+}
+
+cudaError_t launch_concat(const void *Kc, const void *Vc, int units, int cap, int D, int P, int base, int ring,
+                          int ring_head, const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
+                          cudaStream_t stream)
+{
+    if (D == 128)
+        return launch_concat_t<16>(Kc, Vc, units, cap, P, base, ring, ring_head, K_new, V_new, Tq, K_all, V_all, stream);
+    return launch_concat_t<8>(Kc, Vc, units, cap, P, base, ring, ring_head, K_new, V_new, Tq, K_all, V_all, stream);
 }
 
 }  // namespace ec

@@ -79,10 +79,10 @@ class ElasticCacheSession:
         the new rows under the new tokens' queries, then selection and merge over the concatenation.
         Returns a new session holding the compacted result (this one is left untouched)."""
         N, H, Tq, D = Q_new.shape
-        idx = torch.tensor(self.logical_slots(), dtype=torch.long, device=self.device)
-        K_all = torch.cat([self.Kc.index_select(2, idx), K_new], dim=2).contiguous()
-        V_all = torch.cat([self.Vc.index_select(2, idx), V_new], dim=2).contiguous()
-        P = idx.numel()
+        P = self.cache.len
+        K_all = torch.empty((N, H, P + Tq, D), dtype=torch.bfloat16, device=self.device)
+        V_all = torch.empty_like(K_all)
+        ec.ec_cache_concat(self.cache, K_new, V_new, K_all, V_all)
         nxt = ElasticCacheSession(N, H, P + Tq, D, keep_ratio, self.offset, self.scale, self.population,
                                   self.protect_ends, device=self.device)
         ws = torch.empty(ec.ec_importance_workspace(N, H, Tq, D), dtype=torch.uint8, device=self.device)

@@ -595,6 +595,57 @@ def test_second_instruction_on_top_of_a_decoded_cache():
         assert_bf16_close(out, want, f"decode after the second instruction, step {s}")
 
 
+@pytest.mark.parametrize("N,H,D,C,len0,offset,steps,Tq", [
+    (2, 3, 128, 40, 40, 16, 23, 50),      # full cache, ring rotated by 23 mod 16
+    (1, 5, 64, 33, 33, 7, 14, 1),         # whole turns of the ring (14 = 2 * 7), one new row
+    (1, 4, 128, 48, 20, 16, 11, 30),      # still below its budget: no ring yet
+    (2, 2, 64, 24, 10, 23, 40, 9),        # grows to the budget, then evicts; offset = budget - 1
+])
+def test_cache_concat_restores_queue_order(N, H, D, C, len0, offset, steps, Tq):
+    """ec_cache_concat after a decode chain: the oracle's queue (oldest first), then the new rows, bit for bit."""
+    rng = np.random.default_rng(1000 + C + steps)
+    scale = 1.0 / math.sqrt(D)
+    K0b, V0b = rand_bits(rng, (N, H, len0, D)), rand_bits(rng, (N, H, len0, D))
+    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=C + 1)
+    Kc = torch.zeros((N, H, C, D), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    Kc[:, :, :len0], Vc[:, :, :len0] = dev_bf16(K0b), dev_bf16(V0b)
+    cache = ec.ec_cache_init(Kc, Vc, len0, C, offset)
+    ws = scratch(ec.ec_decode_workspace(cache))
+    qb, kb, vb = (rand_bits(rng, (steps, N, H, D)) for _ in range(3))
+    for s in range(steps):
+        queue.step(qb[s], kb[s], vb[s], scale, policy=orc.POLICY_FIXED, budget=C, offset=offset)
+    out = torch.empty((steps, N, H, D), dtype=torch.bfloat16, device="cuda")
+    ec.ec_decode_steps(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), cache, scale, out, ws)
+    P = cache.len
+    assert P == queue.len == min(C, len0 + steps)
+    Knb, Vnb = rand_bits(rng, (N, H, Tq, D)), rand_bits(rng, (N, H, Tq, D))
+    K_all = Guarded((N, H, P + Tq, D), torch.bfloat16, fill=float("nan"))
+    V_all = Guarded((N, H, P + Tq, D), torch.bfloat16, fill=float("nan"))
+    ec.ec_cache_concat(cache, dev_bf16(Knb), dev_bf16(Vnb), K_all.t, V_all.t)
+    K_all.check("K_all")
+    V_all.check("V_all")
+    want_K = np.concatenate([orc.round_bf16(queue.K[:, :P].reshape(N, H, P, D)), Knb], 2)
+    want_V = np.concatenate([orc.round_bf16(queue.V[:, :P].reshape(N, H, P, D)), Vnb], 2)
+    np.testing.assert_array_equal(host_bits(K_all.t), want_K)
+    np.testing.assert_array_equal(host_bits(V_all.t), want_V)
+
+
+def test_cache_concat_rejects_the_ratio_policy_and_bad_shapes():
+    N, H, D, C = 1, 2, 64, 16
+    Kc = torch.zeros((N, H, C + 8, D), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    new = torch.zeros((N, H, 4, D), dtype=torch.bfloat16, device="cuda")
+    all_ = torch.zeros((N, H, C + 4, D), dtype=torch.bfloat16, device="cuda")
+    ratio_cache = ec.ec_cache_init_ratio(Kc, Vc, C, 4, 0.5, 32)
+    with pytest.raises(ec.EcError) as e:
+        ec.ec_cache_concat(ratio_cache, new, new, all_, all_.clone())
+    assert e.value.status == ec.EC_ERR_ARG
+    fixed = ec.ec_cache_init(Kc, Vc, C, C, 4)
+    with pytest.raises(ValueError):
+        ec.ec_cache_concat(fixed, new, new, all_[:, :, :-1].contiguous(), all_[:, :, :-1].contiguous())
+
+
 # ---------------------------------------------------------------- host-resident tensors
 
 def test_host_entry_points_match_the_device_path():
