@@ -21,6 +21,8 @@
  *  - Eq. 3: plain mean over the bucket, the anchor's own vector included.
  *  - Fixed-point elimination: after appending the new row, the row that has exactly
  *    `offset` rows behind it is deleted (Algorithm 1's fix_idx with P = -offset).
+ *  - Mean, maximum and moving-average importance (named in Sec. 3.2 without formulas): the
+ *    definitions written above eco_importance_statistic.
  */
 #include <math.h>
 #include <stdint.h>
@@ -166,6 +168,68 @@ void eco_importance_prefix(const uint16_t *Q, const uint16_t *K, int U, int Tq, 
         free(k);
         free(s);
     }
+}
+
+/*
+ * Other statistics of the attention a key receives (Sec. 3.2 "Importance Metrics" lists summation,
+ * moving average, maximum value and mean; the ablation on the importance metric compares moving
+ * average, mean and sum). The paper prints no formulas for them; the readings taken here:
+ *   stat 0  sum             I[n] = sum_m A[m][n]                            (eco_importance_prefix)
+ *   stat 1  mean            I[n] = (sum_m A[m][n]) / #{queries m that can see key n}
+ *   stat 2  maximum         I[n] = max_m A[m][n]
+ *   stat 3  moving average  E starts at zero; after each query m, in order,
+ *                           E[n] <- beta*E[n] + (1-beta)*A[m][n] for every key n
+ *                           (A[m][n] = 0 for keys the query cannot see); I = E after the last query
+ * Same geometry as eco_importance_prefix: Tq queries, P + Tq keys, query m sees keys n <= m + P.
+ * Q: bf16 [U, Tq, D]; K: bf16 [U, P+Tq, D]; scores [U, P+Tq]. beta is read for stat 3 only.
+ * Returns 0, or -1 for an unknown stat.
+ */
+int eco_importance_statistic(const uint16_t *Q, const uint16_t *K, int U, int Tq, int P, int D, double scale,
+                             int stat, double beta, double *scores)
+{
+    if (stat < 0 || stat > 3) return -1;
+    const int Tk = P + Tq;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < U; ++u) {
+        double *q = (double *)malloc(sizeof(double) * (size_t)Tq * D);
+        double *k = (double *)malloc(sizeof(double) * (size_t)Tk * D);
+        double *a = (double *)malloc(sizeof(double) * (size_t)Tk);
+        eco_widen_bf16(Q + (size_t)u * Tq * D, (int64_t)Tq * D, q);
+        eco_widen_bf16(K + (size_t)u * Tk * D, (int64_t)Tk * D, k);
+        double *I = scores + (size_t)u * Tk;
+        for (int n = 0; n < Tk; ++n) I[n] = 0.0;
+        for (int m = 0; m < Tq; ++m) {
+            const int last = m + P;
+            /* row m of A (Eq. 1), zero past the causal limit */
+            double mx = -INFINITY;
+            for (int n = 0; n <= last; ++n) {
+                double dot = 0.0;
+                for (int c = 0; c < D; ++c) dot += q[(size_t)m * D + c] * k[(size_t)n * D + c];
+                a[n] = scale * dot;
+                if (a[n] > mx) mx = a[n];
+            }
+            double Z = 0.0;
+            for (int n = 0; n <= last; ++n) Z += exp(a[n] - mx);
+            for (int n = 0; n <= last; ++n) a[n] = exp(a[n] - mx) / Z;
+            for (int n = last + 1; n < Tk; ++n) a[n] = 0.0;
+            /* fold the row into the statistic */
+            for (int n = 0; n < Tk; ++n) {
+                if (stat == 0 || stat == 1) I[n] += a[n];
+                else if (stat == 2) { if (a[n] > I[n]) I[n] = a[n]; }
+                else I[n] = beta * I[n] + (1.0 - beta) * a[n];
+            }
+        }
+        if (stat == 1)
+            for (int n = 0; n < Tk; ++n) {
+                int seen_by = 0;                         /* queries m with n <= m + P */
+                for (int m = 0; m < Tq; ++m) if (n <= m + P) ++seen_by;
+                I[n] /= (double)seen_by;
+            }
+        free(q);
+        free(k);
+        free(a);
+    }
+    return 0;
 }
 
 /* Layer-wise population: the mean over the heads of a layer. scores [N, H, T] -> out [N, T]. */

@@ -28,6 +28,9 @@ _lib.eco_keep_count.restype = C.c_int
 _lib.eco_keep_count.argtypes = [C.c_int, C.c_double]
 _lib.eco_importance.restype = None
 _lib.eco_importance.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_double, _f64p, _f64p]
+_lib.eco_importance_statistic.restype = C.c_int
+_lib.eco_importance_statistic.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, C.c_int,
+                                          C.c_double, _f64p]
 _lib.eco_importance_prefix.restype = None
 _lib.eco_importance_prefix.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _f64p, _f64p]
 _lib.eco_layer_mean.restype = None
@@ -95,6 +98,26 @@ def importance_prefix(Q: np.ndarray, K: np.ndarray, scale: float) -> Tuple[np.nd
     lse = np.empty(Q.shape[:-1], np.float64)
     _lib.eco_importance_prefix(_p(Q, _u16p), _p(K, _u16p), U, Tq, P, D, float(scale), _p(scores, _f64p), _p(lse, _f64p))
     return scores, lse
+
+
+STAT_SUM, STAT_MEAN, STAT_MAX, STAT_MOVING_AVERAGE = 0, 1, 2, 3
+
+
+def importance_statistic(Q: np.ndarray, K: np.ndarray, scale: float, stat: int, beta: float = 0.0) -> np.ndarray:
+    """Sum, mean, maximum or moving average (factor beta) of the attention each key receives
+    (Sec. 3.2 "Importance Metrics"). Q uint16 [..., Tq, D], K uint16 [..., P+Tq, D].
+    Returns scores [..., P+Tq] in float64."""
+    Q, K = _bits(Q), _bits(K)
+    assert Q.shape[:-2] == K.shape[:-2] and Q.shape[-1] == K.shape[-1] and K.shape[-2] >= Q.shape[-2]
+    Tq, D = Q.shape[-2:]
+    P = K.shape[-2] - Tq
+    U = int(np.prod(Q.shape[:-2], dtype=np.int64))
+    scores = np.empty(K.shape[:-1], np.float64)
+    rc = _lib.eco_importance_statistic(_p(Q, _u16p), _p(K, _u16p), U, Tq, P, D, float(scale), int(stat), float(beta),
+                                       _p(scores, _f64p))
+    if rc != 0:
+        raise ValueError("unknown statistic")
+    return scores
 
 
 def layer_mean(scores: np.ndarray) -> np.ndarray:

@@ -365,3 +365,70 @@ def test_importance_prefix_matches_library_softmax_and_reduces_to_plain():
             s0, l0 = orc.importance(qb, kb, 0.4)
             np.testing.assert_array_equal(scores, s0)
             np.testing.assert_array_equal(lse, l0)
+
+
+# ------------------------------------------------------------------ other importance statistics (Sec. 3.2)
+
+def _attention_rows(qb, kb, scale):
+    """A [U, Tq, P+Tq] from library routines (fp64 matmul + softmax), zero past the causal limit."""
+    q = torch.from_numpy(wl.bf16_bits_to_f64(qb))
+    k = torch.from_numpy(wl.bf16_bits_to_f64(kb))
+    Tq, Tk = q.shape[-2], k.shape[-2]
+    logits = scale * q @ k.transpose(-1, -2)
+    m_idx, n_idx = torch.arange(Tq)[:, None], torch.arange(Tk)[None, :]
+    logits = logits.masked_fill(n_idx > m_idx + (Tk - Tq), float("-inf"))
+    return torch.softmax(logits, dim=-1)
+
+
+def test_statistics_hand_example():
+    # two tokens, one dimension, q = 1, k = (0, 1), scale = ln 2: A = [[1, 0], [1/3, 2/3]]
+    q = _bf16(np.ones((1, 2, 1)))
+    k = _bf16(np.array([0.0, 1.0]).reshape(1, 2, 1))
+    sc = math.log(2.0)
+    np.testing.assert_allclose(orc.importance_statistic(q, k, sc, orc.STAT_SUM)[0], [4 / 3, 2 / 3], rtol=1e-14)
+    np.testing.assert_allclose(orc.importance_statistic(q, k, sc, orc.STAT_MEAN)[0], [2 / 3, 2 / 3], rtol=1e-14)
+    np.testing.assert_allclose(orc.importance_statistic(q, k, sc, orc.STAT_MAX)[0], [1.0, 2 / 3], rtol=1e-14)
+    # beta = 1/4: E = (3/4, 0) after the first query, then (1/4)(3/4) + (3/4)(1/3) = 7/16 and (3/4)(2/3) = 1/2
+    np.testing.assert_allclose(orc.importance_statistic(q, k, sc, orc.STAT_MOVING_AVERAGE, 0.25)[0], [7 / 16, 1 / 2],
+                               rtol=1e-14)
+
+
+def test_statistics_uniform_attention_closed_forms():
+    # zero queries: A[m][n] = 1/(m + P + 1) for n <= m + P
+    Tq, P, D, beta = 9, 4, 4, Fraction(2, 3)
+    rng = np.random.default_rng(5)
+    q = _bf16(np.zeros((1, Tq, D)))
+    k = _rand_bits(rng, (1, P + Tq, D))
+    first = [max(0, n - P) for n in range(P + Tq)]                      # first query that sees key n
+    mean = [sum(Fraction(1, m + P + 1) for m in range(first[n], Tq)) / (Tq - first[n]) for n in range(P + Tq)]
+    mx = [Fraction(1, first[n] + P + 1) for n in range(P + Tq)]         # the earliest visible row is the largest
+    ema = [sum((1 - beta) * beta ** (Tq - 1 - m) * Fraction(1, m + P + 1) for m in range(first[n], Tq))
+           for n in range(P + Tq)]
+    for stat, want, b in [(orc.STAT_MEAN, mean, 0.0), (orc.STAT_MAX, mx, 0.0), (orc.STAT_MOVING_AVERAGE, ema, float(beta))]:
+        got = orc.importance_statistic(q, k, 0.9, stat, b)[0]
+        np.testing.assert_allclose(got, [float(w) for w in want], rtol=1e-13)
+
+
+@pytest.mark.parametrize("Tq,P,D", [(1, 0, 4), (6, 0, 4), (13, 7, 8), (4, 30, 8)])
+def test_statistics_match_library_softmax(Tq, P, D):
+    rng = np.random.default_rng(Tq * 10 + P)
+    qb, kb = _rand_bits(rng, (3, Tq, D)), _rand_bits(rng, (3, P + Tq, D))
+    A = _attention_rows(qb, kb, 0.5)                                    # [3, Tq, P+Tq]
+    total = A.sum(dim=-2).numpy()
+    np.testing.assert_array_equal(orc.importance_statistic(qb, kb, 0.5, orc.STAT_SUM),
+                                  orc.importance_prefix(qb, kb, 0.5)[0])
+    seen_by = (torch.arange(P + Tq)[None, :] <= torch.arange(Tq)[:, None] + P).sum(dim=0).numpy()
+    np.testing.assert_allclose(orc.importance_statistic(qb, kb, 0.5, orc.STAT_MEAN), total / seen_by, rtol=1e-12)
+    np.testing.assert_allclose(orc.importance_statistic(qb, kb, 0.5, orc.STAT_MAX), A.max(dim=-2).values.numpy(),
+                               rtol=1e-12)
+    beta = 0.8
+    w = (1 - beta) * beta ** torch.arange(Tq - 1, -1, -1, dtype=torch.float64)   # weight of query m at the end
+    want = (w[None, :, None] * A).sum(dim=-2).numpy()
+    got = orc.importance_statistic(qb, kb, 0.5, orc.STAT_MOVING_AVERAGE, beta)
+    np.testing.assert_allclose(got, want, rtol=1e-12)
+    np.testing.assert_allclose(got.sum(-1), 1 - beta ** Tq, rtol=1e-12)          # rows of A carry unit mass
+    # beta = 0 keeps only the last query's row
+    np.testing.assert_allclose(orc.importance_statistic(qb, kb, 0.5, orc.STAT_MOVING_AVERAGE, 0.0),
+                               A[:, -1, :].numpy(), rtol=1e-12)
+    with pytest.raises(ValueError):
+        orc.importance_statistic(qb, kb, 0.5, 7)
