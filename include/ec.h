@@ -110,6 +110,29 @@ int ec_importance_prefix(const void *Q_dev, const void *K_dev, float *scores_dev
                          void *ws_dev, size_t ws_bytes, void *stream);
 
 /*
+ * Other statistics of the attention a key receives (Sec. 3.2 "Importance Metrics" names
+ * summation, moving average, maximum value and mean; the ablation on the importance metric
+ * compares moving average, mean and sum). The paper gives no formulas; with A as in Eq. 1 and
+ * the geometry of ec_importance_prefix (Tq queries, P + Tq keys, query m sees keys n <= m + P):
+ *   EC_STAT_SUM             scores[n] = sum_m A[m][n]          (= ec_importance_prefix)
+ *   EC_STAT_MEAN            the sum divided by the number of queries that can see key n,
+ *                           Tq - max(0, n - P)
+ *   EC_STAT_MAX             scores[n] = max_m A[m][n]
+ *   EC_STAT_MOVING_AVERAGE  E <- beta*E + (1-beta)*A[m][.] over the queries in order, from
+ *                           E = 0; scores = E after the last query, i.e. the sum with query m
+ *                           weighted by (1-beta)*beta^(Tq-1-m). 0 < beta < 1; weights below
+ *                           about 2^-125 count as zero
+ * Arguments as ec_importance_prefix; `beta` is read for the moving average only. lse_dev, when
+ * given, receives the plain log-sum-exp whatever the statistic. The statistic only changes
+ * the scores: selection and merging take them as they take the sum.
+ */
+typedef enum { EC_STAT_SUM = 0, EC_STAT_MEAN = 1, EC_STAT_MAX = 2, EC_STAT_MOVING_AVERAGE = 3 } ec_statistic;
+
+int ec_importance_statistic(const void *Q_dev, const void *K_dev, float *scores_dev, float *lse_dev,
+                            int N, int H, int Tq, int P, int D, float scale, int statistic, double beta,
+                            void *ws_dev, size_t ws_bytes, void *stream);
+
+/*
  * The same importance when the caller already holds every query row's log-sum-exp, as a
  * prefill attention kernel produces it (the paper takes the attention probabilities from
  * the model's own forward pass, Algorithm 1 "Input"): only the column-sum pass runs, which

@@ -19,11 +19,12 @@ LIB_PATH = os.path.join(_PKG, "libec.so")
 EC_OK, EC_ERR_NULL, EC_ERR_SHAPE, EC_ERR_ALIGN, EC_ERR_ARG = 0, 1, 2, 3, 4
 EC_ERR_WORKSPACE, EC_ERR_CUDA, EC_ERR_TIMEOUT, EC_ERR_TOO_LARGE = 5, 6, 7, 8
 EC_PER_HEAD = 0
+EC_STAT_SUM, EC_STAT_MEAN, EC_STAT_MAX, EC_STAT_MOVING_AVERAGE = 0, 1, 2, 3
 EC_LAYER_SHARED = 1
 
 EXPORTS = (
     "ec_status_string", "ec_keep_count",
-    "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_from_lse", "ec_device_status", "ec_selftest_wait_timeout",
+    "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_statistic", "ec_importance_from_lse", "ec_device_status", "ec_selftest_wait_timeout",
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
     "ec_cache_init", "ec_cache_init_ratio", "ec_cache_concat", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc", "ec_compress_host", "ec_decode_steps_host",
@@ -69,6 +70,8 @@ def lib() -> C.CDLL:
     L.ec_importance.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
     L.ec_importance_prefix.restype = i
     L.ec_importance_prefix.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
+    L.ec_importance_statistic.restype = i
+    L.ec_importance_statistic.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, C.c_double, vp, sz, vp]
     L.ec_importance_from_lse.restype = i
     L.ec_importance_from_lse.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
     L.ec_device_status.restype = i
@@ -157,6 +160,17 @@ def ec_importance_prefix(Q: torch.Tensor, K: torch.Tensor, scores: torch.Tensor,
     st = lib().ec_importance_prefix(_ptr(Q), _ptr(K), _ptr(scores), _ptr(lse), N, H, Tq, P, D, float(scale),
                                     _ptr(ws), ws.numel() * ws.element_size(), _stream())
     _check(st, "ec_importance_prefix")
+
+
+def ec_importance_statistic(Q: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, lse: Optional[torch.Tensor],
+                            scale: float, statistic: int, beta: float, ws: torch.Tensor) -> None:
+    """ec_importance_prefix with the statistic chosen: EC_STAT_SUM, EC_STAT_MEAN, EC_STAT_MAX or
+    EC_STAT_MOVING_AVERAGE (factor 0 < beta < 1). Shapes as ec_importance_prefix."""
+    N, H, Tq, D = Q.shape
+    P = K.shape[2] - Tq
+    st = lib().ec_importance_statistic(_ptr(Q), _ptr(K), _ptr(scores), _ptr(lse), N, H, Tq, P, D, float(scale),
+                                       int(statistic), float(beta), _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_importance_statistic")
 
 
 def ec_importance_from_lse(Q: torch.Tensor, K: torch.Tensor, lse: torch.Tensor, scores: torch.Tensor,

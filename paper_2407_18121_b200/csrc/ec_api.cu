@@ -69,23 +69,33 @@ int ec_importance(const void *Q, const void *K, float *scores, float *lse, int N
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || (lse && !aligned(lse, 16))) return EC_ERR_ALIGN;
     if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EC_ERR_ALIGN;
-    cudaError_t e = ec::launch_importance(Q, K, scores, lse, nullptr, N, H, T, 0, D, scale, ws, (cudaStream_t)stream);
+    cudaError_t e = ec::launch_importance(Q, K, scores, lse, nullptr, N, H, T, 0, D, scale, EC_STAT_SUM, 0.0, ws,
+                                          (cudaStream_t)stream);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 
-int ec_importance_prefix(const void *Q, const void *K, float *scores, float *lse, int N, int H, int Tq, int P, int D,
-                         float scale, void *ws, size_t ws_bytes, void *stream)
+int ec_importance_statistic(const void *Q, const void *K, float *scores, float *lse, int N, int H, int Tq, int P, int D,
+                            float scale, int statistic, double beta, void *ws, size_t ws_bytes, void *stream)
 {
     if (!Q || !K || !scores) return EC_ERR_NULL;
     if (P < 0 || Tq < 1 || (long long)P + Tq > kMaxT) return EC_ERR_SHAPE;
     int st = check_shape(N, H, Tq + P, D);
     if (st != EC_OK) return st;
     if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
+    if (statistic < EC_STAT_SUM || statistic > EC_STAT_MOVING_AVERAGE) return EC_ERR_ARG;
+    if (statistic == EC_STAT_MOVING_AVERAGE && !(beta > 0.0 && beta < 1.0)) return EC_ERR_ARG;
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || (lse && !aligned(lse, 16))) return EC_ERR_ALIGN;
     if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, Tq, D)) return EC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EC_ERR_ALIGN;
-    cudaError_t e = ec::launch_importance(Q, K, scores, lse, nullptr, N, H, Tq, P, D, scale, ws, (cudaStream_t)stream);
+    cudaError_t e = ec::launch_importance(Q, K, scores, lse, nullptr, N, H, Tq, P, D, scale, statistic, beta, ws,
+                                          (cudaStream_t)stream);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+int ec_importance_prefix(const void *Q, const void *K, float *scores, float *lse, int N, int H, int Tq, int P, int D,
+                         float scale, void *ws, size_t ws_bytes, void *stream)
+{
+    return ec_importance_statistic(Q, K, scores, lse, N, H, Tq, P, D, scale, EC_STAT_SUM, 0.0, ws, ws_bytes, stream);
 }
 
 int ec_importance_from_lse(const void *Q, const void *K, const float *lse, float *scores, int N, int H, int T, int D,
@@ -98,7 +108,8 @@ int ec_importance_from_lse(const void *Q, const void *K, const float *lse, float
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || !aligned(lse, 4)) return EC_ERR_ALIGN;
     if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EC_ERR_ALIGN;
-    cudaError_t e = ec::launch_importance(Q, K, scores, nullptr, lse, N, H, T, 0, D, scale, ws, (cudaStream_t)stream);
+    cudaError_t e = ec::launch_importance(Q, K, scores, nullptr, lse, N, H, T, 0, D, scale, EC_STAT_SUM, 0.0, ws,
+                                          (cudaStream_t)stream);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 

@@ -57,7 +57,8 @@ __device__ __forceinline__ float fast_exp2(float x)
 
 // ---- launchers implemented in the .cu files (all asynchronous on `stream`) ----
 cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out, const float *lse_in,
-                              int N, int H, int Tq, int P, int D, float scale, void *ws, cudaStream_t stream);
+                              int N, int H, int Tq, int P, int D, float scale, int statistic, double beta, void *ws,
+                              cudaStream_t stream);
 size_t importance_workspace_bytes(int N, int H, int T, int D);
 cudaError_t launch_wait_selftest(void *ws, unsigned limit_us, cudaStream_t stream);
 

@@ -217,16 +217,31 @@ struct Geometry {
     __host__ __device__ int imin(int j) const { int d = j * kTileRows - P; return d > 0 ? d / kTileRows : 0; }
 };
 
-// PASS2 == false: stationary = query tile i, streamed = key tiles jmax(i) .. 0      -> lse2 (and lse_out)
-// PASS2 == true : stationary = key tile j,   streamed = query tiles imin(j) .. ntq-1 -> scores
+// How the attention rows are folded into a per-key statistic (Sec. 3.2 "Importance Metrics").
+// Query m enters pass 2 with weight 2^(wa + wb*m): pass 1 stores lse - (wa + wb*m), so the weight
+// costs nothing per element. wa = wb = 0 is the plain sum; a moving average with factor beta is
+// wa = log2(1-beta) + (Tq-1)*log2(beta), wb = -log2(beta). `mean` divides each key's total by the
+// number of queries that can see it.
+struct Fold {
+    float wa, wb;
+    int mean;
+};
+
+constexpr int kPass1 = 0, kPass2Sum = 1, kPass2Max = 2;
+
+// MODE kPass1:    stationary = query tile i, streamed = key tiles jmax(i) .. 0      -> lse2 (and lse_out)
+// MODE kPass2Sum: stationary = key tile j,   streamed = query tiles imin(j) .. ntq-1 -> scores (weighted sums)
+// MODE kPass2Max: the same walk, keeping the maximum over the queries instead of the sum
 // A streamed tile needs the mask only when 128*(i-j) + P < 127. lse2 is padded to ntq*128 entries
 // per unit; entries past Tq hold +inf so that pass 2 gives those (non-existent) queries zero weight.
-template <int D, int STAGES, bool PASS2>
+template <int D, int STAGES, int MODE>
 __global__ void __launch_bounds__(kThreads, 2)
 importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const Geometry geo, int n_super, float c, float *__restrict__ lse2, float *__restrict__ lse_out,
-                  float *__restrict__ scores, int *__restrict__ status)
+                  const Geometry geo, const Fold fold, int n_super, float c, float *__restrict__ lse2,
+                  float *__restrict__ lse_out, float *__restrict__ scores, int *__restrict__ status)
 {
+    constexpr bool PASS2 = MODE != kPass1;
+    constexpr bool TAKE_MAX = MODE == kPass2Max;
     using L = Smem<D, STAGES>;
     constexpr int kTileBytes = L::kTileBytes;
     constexpr int kBoxes = D / 64;                          // TMA boxes (64 bf16 = 128 B wide) per tile
@@ -449,8 +464,13 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                     if (i4 * 4 + 2 < lim) p2 = 0.f;
                                     if (i4 * 4 + 3 < lim) p3 = 0.f;
                                 }
-                                accA = __fadd2_rn(accA, make_float2(p0, p1));
-                                accB = __fadd2_rn(accB, make_float2(p2, p3));
+                                if constexpr (TAKE_MAX) {
+                                    accA.x = fmaxf(accA.x, p0); accA.y = fmaxf(accA.y, p1);
+                                    accB.x = fmaxf(accB.x, p2); accB.y = fmaxf(accB.y, p3);
+                                } else {
+                                    accA = __fadd2_rn(accA, make_float2(p0, p1));
+                                    accB = __fadd2_rn(accB, make_float2(p2, p3));
+                                }
                             }
                         }
                     };
@@ -477,9 +497,11 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
                 // the two halves of a row meet: the second-half thread hands its result over
                 const uint32_t iph = it & 1u;
+                const float own = TAKE_MAX ? fmaxf(fmaxf(accA.x, accA.y), fmaxf(accB.x, accB.y))
+                                           : (accA.x + accA.y) + (accB.x + accB.y);
                 if (half == 1) {
                     if (!mbar_wait(bar_comb_empty, iph ^ 1u, abort_flag, status)) { alive = false; break; }
-                    comb_s[r] = PASS2 ? make_float2((accA.x + accA.y) + (accB.x + accB.y), 0.f) : make_float2(mrun, Z);
+                    comb_s[r] = PASS2 ? make_float2(own, 0.f) : make_float2(mrun, Z);
                     mbar_arrive(bar_comb_full);
                 } else {
                     if (!mbar_wait(bar_comb_full, iph, abort_flag, status)) { alive = false; break; }
@@ -490,10 +512,12 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         const float M = fmaxf(mrun, o.x);             // finite: column 0 of some tile is visible
                         const float Zs = Z * fast_exp2(mrun - M) + o.y * fast_exp2(o.x - M);
                         const float l2 = (row < geo.Tq) ? M + __log2f(Zs) : INFINITY;
-                        lse2[lse_row + row] = l2;
+                        lse2[lse_row + row] = l2 - (fold.wa + fold.wb * (float)row);   // +inf stays +inf
                         if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
                     } else if (row < Tk) {
-                        scores[(size_t)unit * Tk + row] = ((accA.x + accA.y) + (accB.x + accB.y)) + o.x;
+                        float total = TAKE_MAX ? fmaxf(own, o.x) : own + o.x;
+                        if (fold.mean) total /= (float)(geo.Tq - (row > geo.P ? row - geo.P : 0));   // queries that see this key
+                        scores[(size_t)unit * Tk + row] = total;
                     }
                 }
                 ++it;
@@ -574,21 +598,30 @@ int sm_count()
 }
 
 template <int D, int STAGES>
-cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int units, const Geometry &geo, float c,
-                          float *lse2, float *lse_out, float *scores, int *status, bool first_pass, cudaStream_t stream)
+cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int units, const Geometry &geo, const Fold &fold,
+                          bool take_max, float c, float *lse2, float *lse_out, float *scores, int *status, bool first_pass,
+                          cudaStream_t stream)
 {
     constexpr int smem = Smem<D, STAGES>::kDynBytes;
-    cudaError_t e = cudaFuncSetAttribute(importance_kernel<D, STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(importance_kernel<D, STAGES, kPass1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(importance_kernel<D, STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(importance_kernel<D, STAGES, kPass2Sum>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(importance_kernel<D, STAGES, kPass2Max>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const long long resident = 2LL * sm_count();              // two persistent CTAs per SM
     const long long super1 = (long long)units * ((geo.ntq + 1) / 2), super2 = (long long)units * ((geo.ntk + 1) / 2);
+    const unsigned grid1 = (unsigned)(super1 < resident ? super1 : resident);
+    const unsigned grid2 = (unsigned)(super2 < resident ? super2 : resident);
     if (first_pass)
-        importance_kernel<D, STAGES, false><<<(unsigned)(super1 < resident ? super1 : resident), kThreads, smem, stream>>>(
-            mq, mk, geo, (int)super1, c, lse2, lse_out, scores, status);
-    importance_kernel<D, STAGES, true><<<(unsigned)(super2 < resident ? super2 : resident), kThreads, smem, stream>>>(
-        mq, mk, geo, (int)super2, c, lse2, lse_out, scores, status);
+        importance_kernel<D, STAGES, kPass1><<<grid1, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)super1, c, lse2,
+                                                                              lse_out, scores, status);
+    if (take_max)
+        importance_kernel<D, STAGES, kPass2Max><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)super2, c, lse2,
+                                                                                 lse_out, scores, status);
+    else
+        importance_kernel<D, STAGES, kPass2Sum><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)super2, c, lse2,
+                                                                                 lse_out, scores, status);
     return cudaGetLastError();
 }
 
@@ -609,10 +642,12 @@ size_t importance_workspace_bytes(int N, int H, int T, int D)
     return kStatusBytes + (size_t)N * H * nt * kTileRows * sizeof(float);   // status block + padded lse
 }
 
-// lse_in == nullptr: both passes. Otherwise the caller's normaliser replaces pass 1.
+// lse_in == nullptr: both passes. Otherwise the caller's normaliser replaces pass 1 (plain sum only).
 // Q: [units, Tq, D]; K: [units, P + Tq, D]; scores: [units, P + Tq]; lse_out / lse_in: [units, Tq].
+// statistic: EC_STAT_*; beta in (0, 1) is read for the moving average only.
 cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out, const float *lse_in,
-                              int N, int H, int Tq, int P, int D, float scale, void *ws, cudaStream_t stream)
+                              int N, int H, int Tq, int P, int D, float scale, int statistic, double beta, void *ws,
+                              cudaStream_t stream)
 {
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return e;
@@ -625,6 +660,12 @@ cudaError_t launch_importance(const void *Q, const void *K, float *scores, float
     geo.ntq = (Tq + kTileRows - 1) / kTileRows;
     geo.ntk = (Tq + P + kTileRows - 1) / kTileRows;
     if ((long long)units * geo.ntk > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    Fold fold = {0.f, 0.f, statistic == EC_STAT_MEAN ? 1 : 0};
+    if (statistic == EC_STAT_MOVING_AVERAGE) {
+        const double lb = log2(beta);
+        fold.wa = (float)(log2(1.0 - beta) + (double)(Tq - 1) * lb);
+        fold.wb = (float)(-lb);
+    }
     CUtensorMap mq, mk;
     if (!make_map(&mq, Q, units, Tq, D) || !make_map(&mk, K, units, Tq + P, D)) return cudaErrorInvalidValue;
     if (lse_in) {
@@ -632,9 +673,12 @@ cudaError_t launch_importance(const void *Q, const void *K, float *scores, float
         lse_import_kernel<<<g, 256, 0, stream>>>(lse_in, lse2, Tq, geo.ntq * kTileRows);
     }
     const float c = scale * kLog2e;
+    const bool take_max = statistic == EC_STAT_MAX;
     if (D == 128)
-        return launch_passes<128, 2>(mq, mk, units, geo, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
-    return launch_passes<64, 4>(mq, mk, units, geo, c, lse2, lse_out, scores, status, lse_in == nullptr, stream);
+        return launch_passes<128, 2>(mq, mk, units, geo, fold, take_max, c, lse2, lse_out, scores, status,
+                                     lse_in == nullptr, stream);
+    return launch_passes<64, 4>(mq, mk, units, geo, fold, take_max, c, lse2, lse_out, scores, status, lse_in == nullptr,
+                                stream);
 }
 
 }  // namespace ec

@@ -519,6 +519,46 @@ def test_importance_prefix_matches_oracle(N, H, Tq, P, D):
     np.testing.assert_allclose(host_f64(scores.t).sum(-1), Tq, rtol=1e-3)
 
 
+# ---------------------------------------------------------------- other importance statistics (Sec. 3.2)
+
+@pytest.mark.parametrize("N,H,Tq,P,D", [(2, 2, 200, 127, 128), (1, 3, 129, 0, 64), (1, 2, 640, 0, 128), (1, 2, 70, 400, 128)])
+@pytest.mark.parametrize("stat,beta", [("mean", 0.0), ("max", 0.0), ("moving_average", 0.9), ("moving_average", 0.99)])
+def test_importance_statistics_match_oracle(N, H, Tq, P, D, stat, beta):
+    rng = np.random.default_rng(7 * Tq + P + len(stat))
+    Qb, Kb = rand_bits(rng, (N, H, Tq, D)), rand_bits(rng, (N, H, P + Tq, D))
+    scale = 1.0 / math.sqrt(D)
+    o_stat = {"mean": orc.STAT_MEAN, "max": orc.STAT_MAX, "moving_average": orc.STAT_MOVING_AVERAGE}[stat]
+    g_stat = {"mean": ec.EC_STAT_MEAN, "max": ec.EC_STAT_MAX, "moving_average": ec.EC_STAT_MOVING_AVERAGE}[stat]
+    want = orc.importance_statistic(Qb, Kb, scale, o_stat, beta)
+    _, want_lse = orc.importance_prefix(Qb, Kb, scale)
+    scores = Guarded((N, H, P + Tq), torch.float32, fill=float("nan"))
+    lse = Guarded((N, H, Tq), torch.float32, fill=float("nan"))
+    ws = scratch(ec.ec_importance_workspace(N, H, Tq, D))
+    ec.ec_importance_statistic(dev_bf16(Qb), dev_bf16(Kb), scores.t, lse.t, scale, g_stat, beta, ws)
+    assert ec.ec_device_status(ws) == ec.EC_OK
+    scores.check("scores")
+    lse.check("lse")
+    assert_rel_close(scores.t, want, SCORE_RTOL, what=f"{stat} importance")
+    assert_rel_close(lse.t, want_lse, 1e-3, atol=1e-3, what="lse is the plain one whatever the statistic")
+
+
+def test_importance_statistic_sum_is_the_prefix_call_and_bad_arguments_are_refused():
+    rng = np.random.default_rng(3)
+    N, H, Tq, P, D = 1, 2, 150, 20, 128
+    Qb, Kb = rand_bits(rng, (N, H, Tq, D)), rand_bits(rng, (N, H, P + Tq, D))
+    Q, K = dev_bf16(Qb), dev_bf16(Kb)
+    a = torch.empty((N, H, P + Tq), dtype=torch.float32, device="cuda")
+    b = torch.empty_like(a)
+    ws = scratch(ec.ec_importance_workspace(N, H, Tq, D))
+    ec.ec_importance_prefix(Q, K, a, None, 0.1, ws)
+    ec.ec_importance_statistic(Q, K, b, None, 0.1, ec.EC_STAT_SUM, 0.0, ws)
+    assert torch.equal(a, b)
+    for stat, beta in [(ec.EC_STAT_MOVING_AVERAGE, 0.0), (ec.EC_STAT_MOVING_AVERAGE, 1.0), (4, 0.5), (-1, 0.5)]:
+        with pytest.raises(ec.EcError) as e:
+            ec.ec_importance_statistic(Q, K, b, None, 0.1, stat, beta, ws)
+        assert e.value.status == ec.EC_ERR_ARG
+
+
 # ---------------------------------------------------------------- failure path of the bounded waits
 
 def test_bounded_wait_expires_reports_and_leaves_the_context_usable():
