@@ -175,6 +175,7 @@ def run_reference(args, w: wl.Workload):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    from oracle import ec_oracle as orc
     per_step = []
     info = None
     for i in range(args.warmup + args.steps):
@@ -187,7 +188,7 @@ def run_reference(args, w: wl.Workload):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(w),
+            "config": workload_config(w, orc.keep_count(w.prompt_len, w.keep_ratio)),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
                              "sample": info["sample"]},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -195,11 +196,27 @@ def run_reference(args, w: wl.Workload):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(w: wl.Workload):
+def workload_config(w: wl.Workload, n_keep: int):
     return {"workload": w.name, "batch": w.batch, "layers": w.layers, "heads": w.heads, "head_dim": w.head_dim,
             "prompt_len": w.prompt_len, "keep_ratio": w.keep_ratio, "decode_steps": w.decode_steps,
-            "offset": w.offset, "population": "per_head", "protect_ends": True,
-            "l2": "inputs larger than L2 (prompt Q/K/V and the compacted cache each exceed 126 MB per pass)"}
+            "offset": w.offset, "population": "per_head", "protect_ends": True, "l2": l2_statement(w, n_keep)}
+
+
+L2_BYTES = 126e6
+
+
+def l2_statement(w: wl.Workload, n_keep: int) -> str:
+    """Whether the data each timed stage streams exceeds the 126 MB L2 (nothing is flushed between passes)."""
+    units = w.N * w.heads
+    prompt = units * w.prompt_len * w.head_dim * 2                    # each of Q, K, V
+    cache = 2 * units * n_keep * w.head_dim * 2                       # K and V rows read by every decode step
+    if prompt > L2_BYTES and cache > L2_BYTES:
+        return (f"inputs larger than L2 (prompt Q, K, V {prompt / 1e6:.0f} MB each and the compacted cache "
+                f"{cache / 1e6:.0f} MB per step exceed 126 MB)")
+    small = [n for n, b in (("prompt tensors", prompt), ("compacted cache", cache)) if b <= L2_BYTES]
+    return (f"NOT larger than L2: {' and '.join(small)} fit the 126 MB L2 (prompt {prompt / 1e6:.0f} MB per tensor, "
+            f"cache {cache / 1e6:.0f} MB), so the bandwidth figures of this workload are L2-assisted")
+
 
 
 # ----------------------------------------------------------------------------- rank logic
@@ -383,7 +400,7 @@ def run_ours(args, w: wl.Workload):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "storage_dtype": "bf16", "data": "synthetic",
-        "config": workload_config(w),
+        "config": workload_config(w, ec.ec_keep_count(w.prompt_len, w.keep_ratio)),
         "stages_ms": {"importance": imp_ms, "select_merge": mrg_ms, "decode_loop": dec_ms,
                       "decode_per_token_us": dec_ms * 1e3 / S, "whole_pass_cuda_graph_replay": graph_ms},
         "decode_only_tokens_per_s": w.batch * S * world / (dec_ms * 1e-3),

@@ -76,6 +76,11 @@ WORKLOADS = {
     # long-context stress, heavy-tailed importance
     "long8k": Workload("long8k", 16, 4, 32, 128, 8192, (0.1,), 2048,
                        1.0 / math.sqrt(128.0), 16, 4, "zipf"),
+    # Qwen-VL-7B shapes (Sec. 4.1 names it as the second backbone): 32 layers x 32 heads x 128, 256 image
+    # tokens (its adapter's fixed output length) + 64 text tokens, the paper's recent distance of 25.
+    # Not one of the five measured configurations: an extra parity and timing case.
+    "qwenvl7b_b1": Workload("qwenvl7b_b1", 1, 32, 32, 128, 320, (0.5,), 512,
+                            1.0 / math.sqrt(128.0), 25, 5, "lowrank", n_image=256, rank=8),
 }
 CONFIG_ORDER = ("tiny", "llava7b_b1", "llava7b_b8", "llava13b_b4", "long8k")
 

@@ -98,6 +98,11 @@ def test_7b_batch8_shapes_full_length():
     run_workload(w, [0, 100, 255], [(0, 0), (1, 16), (2, 31)], 40)
 
 
+def test_qwenvl_shapes_full_size():
+    w = wl.WORKLOADS["qwenvl7b_b1"]          # T = 320 (2.5 tiles), 160 kept rows, recent distance 25
+    run_workload(w, list(range(w.N)), [(0, 0), (7, 19), (31, 31)], 60)
+
+
 def test_longest_supported_prompt():
     """T = 16384 (the documented maximum), one unit: 128 tiles per pass in the importance kernels,
     64 KB of keys in the selection kernel's shared memory, 64 slices in the merge kernel."""
