@@ -271,6 +271,24 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int nts = PASS2 ? geo.ntk : geo.ntq;              // stationary tiles per unit
     const int spu = (nts + 1) / 2;                          // item pairs per unit
 
+    // Static schedule: in round k this CTA takes pair k*grid + (cta + k*rot) mod grid, so that a round
+    // covers consecutive pairs (units in order, for L2 reuse). With an odd tile count the unit's
+    // middle tile is a pair of half the cost, and a CTA meets cost classes cta + k*(grid + rot) mod
+    // spu: when grid mod spu shares a factor with spu, some CTAs would never get a cheap pair
+    // (measured: 15% slower at T = 320, 10% at T = 896), so rot then makes (grid + rot) mod spu = 1.
+    // Otherwise rot = 0. Only the last round can be partial.
+    const int grid_n = (int)gridDim.x;
+    int rot = 0;
+    if ((nts & 1) && spu > 1) {
+        int a = grid_n % spu, b = spu;
+        while (a) { const int t = b % a; b = a; a = t; }      // b = gcd(grid mod spu, spu)
+        if (b != 1) rot = ((1 - grid_n) % spu + spu) % spu;
+    }
+    auto pair_of_round = [&](int k) -> int {
+        const long long sidx = (long long)k * grid_n + ((int)blockIdx.x + k * rot) % grid_n;
+        return sidx < n_super ? (int)sidx : -1;
+    };
+
     // a CTA of this launch has already given up: leave at once instead of timing out again
     if (threadIdx.x == 0) *abort_flag = *reinterpret_cast<volatile int *>(status);
     __syncthreads();
@@ -322,7 +340,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t armed = 0;
-            for (int sidx = blockIdx.x; alive && sidx < n_super; sidx += gridDim.x) {
+            for (int round = 0, sidx; alive && (sidx = pair_of_round(round)) >= 0; ++round) {
                 for (int sub = 0; alive && sub < 2; ++sub) {
                     int unit, st, first, count;
                     if (!item_of(sidx, sub, unit, st, first, count)) break;
@@ -355,7 +373,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            for (int sidx = blockIdx.x; alive && sidx < n_super; sidx += gridDim.x) {
+            for (int round = 0, sidx; alive && (sidx = pair_of_round(round)) >= 0; ++round) {
                 for (int sub = 0; alive && sub < 2; ++sub) {
                     int unit, st, first, count;
                     if (!item_of(sidx, sub, unit, st, first, count)) break;
@@ -391,7 +409,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int r = q4 * 32 + lane;                         // row of the stationary tile = TMEM lane
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(half * 64);
         const int Tk = geo.Tk();
-        for (int sidx = blockIdx.x; alive && sidx < n_super; sidx += gridDim.x) {
+        for (int round = 0, sidx; alive && (sidx = pair_of_round(round)) >= 0; ++round) {
             for (int sub = 0; alive && sub < 2; ++sub) {
                 int unit, st, first, count;
                 if (!item_of(sidx, sub, unit, st, first, count)) break;
