@@ -51,3 +51,26 @@ def test_reference_arm_is_silent_on_other_ranks():
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                         "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert p.returncode == 0 and p.stdout.strip() == ""
+
+
+def test_bench_says_per_workload_whether_its_data_exceeds_l2():
+    import bench
+    from oracle import ec_oracle as orc
+    from paper_2407_18121_b200 import workloads as wl
+    big = wl.WORKLOADS["llava7b_b1"]
+    small = wl.WORKLOADS["qwenvl7b_b1"]
+    s_big = bench.l2_statement(big, orc.keep_count(big.prompt_len, big.keep_ratio))
+    s_small = bench.l2_statement(small, orc.keep_count(small.prompt_len, small.keep_ratio))
+    assert s_big.startswith("inputs larger than L2") and "168 MB" in s_big
+    assert s_small.startswith("NOT larger than L2") and "84 MB" in s_small
+
+
+def test_oracle_sample_is_bounded_and_scaled():
+    import bench
+    from paper_2407_18121_b200 import workloads as wl
+    for name, w in wl.WORKLOADS.items():
+        problems, steps = bench.oracle_sample_size(w)
+        assert 1 <= problems <= w.N and 4 <= steps <= w.decode_steps, name
+        # the sampled prompt stage stays within the multiply-add budget unless a single problem exceeds it
+        per_problem = w.heads * w.prompt_len * (w.prompt_len + 1) / 2 * w.head_dim
+        assert problems == 1 or problems * per_problem <= 1.0e11 + per_problem, name
