@@ -40,13 +40,22 @@ __device__ __forceinline__ void transpose32(uint32_t *m)
     uint32_t mask = 0x0000FFFFu;
 #pragma unroll 1
     for (int j = 16; j != 0; j >>= 1) {
-#pragma unroll 4
-        for (int i = 0; i < 16; ++i) {
-            const int k = ((i & ~(j - 1)) << 1) | (i & (j - 1));      // i-th index with bit j clear
-            const uint32_t lo = m[k * 32], hi = m[(k + j) * 32];
-            const uint32_t t = (lo ^ (hi >> j)) & mask;
-            m[k * 32] = lo ^ t;
-            m[(k + j) * 32] = hi ^ (t << j);
+#pragma unroll 1
+        for (int h = 0; h < 16; h += 8) {              // eight word pairs at a time: all loads, then all stores,
+            uint32_t lo[8], hi[8];                      // so that the loads do not queue behind the stores
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int k = (((h + i) & ~(j - 1)) << 1) | ((h + i) & (j - 1));   // (h+i)-th index with bit j clear
+                lo[i] = m[k * 32];
+                hi[i] = m[(k + j) * 32];
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int k = (((h + i) & ~(j - 1)) << 1) | ((h + i) & (j - 1));
+                const uint32_t t = (lo[i] ^ (hi[i] >> j)) & mask;
+                m[k * 32] = lo[i] ^ t;
+                m[(k + j) * 32] = hi[i] ^ (t << j);
+            }
         }
         mask ^= mask << (j >> 1);
     }
@@ -166,34 +175,35 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
 
     const uint32_t lt_mask = (1u << lane) - 1u;
     int32_t *ap0 = anchor_pos + (size_t)unit * replicate * C;
-#pragma unroll 2
-    for (int j = 0; j < kKeysPerLane; ++j) {
+    const int rows = min(kKeysPerLane, (T - base + 31) >> 5);          // rows of this warp that hold positions < T
+#pragma unroll 1
+    for (int j = 0; j < rows; ++j) {
         const bool is_gt = (greater >> j) & 1u, is_eq = (undecided >> j) & 1u;
         const uint32_t bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
         const uint32_t g_here = gb + __popc(bg & lt_mask), e_here = eb + __popc(be & lt_mask);
-        int idx = -1;                                      // anchors before this position = its own index
-        if (is_gt) idx = (int)(g_here + min(e_here, need_eq));
-        else if (is_eq && e_here < need_eq) idx = (int)(g_here + e_here);
-        if (idx >= 0) {
-            const int t = base + 32 * j + lane;
-            for (int r = 0; r < replicate; ++r) ap0[(size_t)r * C + idx] = t;
-        }
+        // anchors before this position = its own index; one predicated store, no divergent code
+        const bool take = is_gt || (is_eq && e_here < need_eq);
+        const int idx = (int)(g_here + min(e_here, need_eq));
+        if (take) ap0[idx] = base + 32 * j + lane;
         gb += __popc(bg);
         eb += __popc(be);
     }
 
     // the merge kernel behind this one may start scheduling; it waits for this grid to finish
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (bucket_len) {
-        // Eq. 2: bucket k spans floor((t_{k-1}+t_k)/2)+1 .. floor((t_k+t_{k+1})/2); the anchors just
-        // written by the unit's own warps are visible after the barrier
+    if (bucket_len || replicate > 1) {
+        // the anchors just written by the unit's own warps are visible after the barrier
         if (G == 1) __syncwarp(); else __syncthreads();
         const volatile int32_t *av = ap0;
         for (int kk = wu * 32 + lane; kk < C; kk += 32 * G) {
             const int c0 = av[kk];
-            const int lo = (kk == 0) ? 0 : ((av[kk - 1] + c0) >> 1) + 1;
-            const int hi = (kk == C - 1) ? T - 1 : ((c0 + av[kk + 1]) >> 1);
-            for (int r = 0; r < replicate; ++r) bucket_len[((size_t)unit * replicate + r) * C + kk] = hi - lo + 1;
+            for (int r = 1; r < replicate; ++r) ap0[(size_t)r * C + kk] = c0;       // shared population: same anchors
+            if (bucket_len) {
+                // Eq. 2: bucket k spans floor((t_{k-1}+t_k)/2)+1 .. floor((t_k+t_{k+1})/2)
+                const int lo = (kk == 0) ? 0 : ((av[kk - 1] + c0) >> 1) + 1;
+                const int hi = (kk == C - 1) ? T - 1 : ((c0 + av[kk + 1]) >> 1);
+                for (int r = 0; r < replicate; ++r) bucket_len[((size_t)unit * replicate + r) * C + kk] = hi - lo + 1;
+            }
         }
     }
 }
