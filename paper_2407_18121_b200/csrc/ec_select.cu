@@ -70,7 +70,8 @@ __device__ __forceinline__ void transpose32(uint32_t *m)
 //     the unit have the bit set, those stay undecided and the others are out; otherwise they are all
 //     anchors (`greater`), `need` shrinks by their count and the others stay undecided. All keys
 //     agree on the bits above the highest bit in which the smallest and the largest key differ, so
-//     the descent starts there. What is still undecided at the end equals the threshold: ties, of
+//     the descent starts there and takes two bits per step (the three counts of a step need one
+//     round of warp reductions). What is still undecided at the end equals the threshold: ties, of
 //     which the `need` lowest positions are taken. Protected positions (first, last) are anchors
 //     from the start.
 //  3. Ordered compaction with warp ballots, one row of 32 consecutive positions at a time.
@@ -80,7 +81,7 @@ __global__ void __launch_bounds__(G == 1 ? 128 : 32 * G)
 select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int protect_ends, int replicate,
               int32_t *__restrict__ anchor_pos, int32_t *__restrict__ bucket_len)
 {
-    __shared__ uint32_t xa[2][kMaxWarpsPerUnit], xb[kMaxWarpsPerUnit];     // cross-warp exchange (G > 1)
+    __shared__ uint32_t xa[2][kMaxWarpsPerUnit], xc[2][kMaxWarpsPerUnit], xb[kMaxWarpsPerUnit];   // cross-warp exchange (G > 1)
     extern __shared__ uint32_t planes_all[];                               // 32 x 32 words per warp
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int unit = (G == 1) ? blockIdx.x * 4 + warp : blockIdx.x;
@@ -102,6 +103,17 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
         for (int w = 0; w < G; ++w) t += xa[par][w];
         par ^= 1;
         return t;
+    };
+    auto unit_sum2 = [&](uint32_t &a, uint32_t &b) {       // two sums for the price of one barrier
+        a = __reduce_add_sync(0xFFFFFFFFu, a);
+        b = __reduce_add_sync(0xFFFFFFFFu, b);
+        if (G == 1) return;
+        if (lane == 0) { xa[par][wu] = a; xc[par][wu] = b; }
+        __syncthreads();
+        a = 0; b = 0;
+#pragma unroll
+        for (int w = 0; w < G; ++w) { a += xa[par][w]; b += xc[par][w]; }
+        par ^= 1;
     };
 
     // pl[(31 - j) * 32] = key of row j, so that after the transpose pl[(31 - b) * 32] is the plane of
@@ -144,9 +156,28 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
         undecided = 0u;                                   // only the protected keys are anchors
     } else if (kmin != kmax) {                            // (kmin == kmax: every unprotected key is a tie)
         const int nbits = 32 - __clz(kmin ^ kmax);
+        int b = nbits - 1;
 #pragma unroll 1
-        for (int b = nbits - 1; b >= 0; --b) {            // uniform over the unit
-            const uint32_t plane = pl[(31 - b) * 32];
+        for (; b >= 1; b -= 2) {                          // two bits per step; uniform over the unit
+            const uint32_t p1 = pl[(31 - b) * 32], p0 = pl[(32 - b) * 32];
+            const uint32_t u11 = undecided & p1 & p0, u10 = undecided & p1 & ~p0, u01 = undecided & ~p1 & p0;
+            // counts of the three non-zero patterns: c11 and c10 share a word (a unit has at most
+            // 16384 keys, so the 16-bit fields cannot carry into each other)
+            uint32_t packed = (uint32_t)__popc(u11) | ((uint32_t)__popc(u10) << 16), c01 = (uint32_t)__popc(u01);
+            unit_sum2(packed, c01);
+            const uint32_t c11 = packed & 0xFFFFu, c10 = packed >> 16;
+            if (c11 >= need) {
+                undecided = u11;
+            } else if (c11 + c10 >= need) {
+                need -= c11; greater |= u11; undecided = u10;
+            } else if (c11 + c10 + c01 >= need) {
+                need -= c11 + c10; greater |= u11 | u10; undecided = u01;
+            } else {
+                need -= c11 + c10 + c01; greater |= u11 | u10 | u01; undecided &= ~(p1 | p0);
+            }
+        }
+        if (b == 0) {                                     // an odd number of bits: the last one alone
+            const uint32_t plane = pl[31 * 32];
             const uint32_t ones = undecided & plane;
             const uint32_t c1 = unit_sum(__popc(ones));
             if (c1 >= need) {
@@ -176,7 +207,7 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
     const uint32_t lt_mask = (1u << lane) - 1u;
     int32_t *ap0 = anchor_pos + (size_t)unit * replicate * C;
     const int rows = min(kKeysPerLane, (T - base + 31) >> 5);          // rows of this warp that hold positions < T
-#pragma unroll 1
+#pragma unroll 4
     for (int j = 0; j < rows; ++j) {
         const bool is_gt = (greater >> j) & 1u, is_eq = (undecided >> j) & 1u;
         const uint32_t bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
