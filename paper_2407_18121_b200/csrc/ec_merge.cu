@@ -48,7 +48,7 @@ __device__ __forceinline__ int first_bucket_from(const int32_t *anch, int C, int
 // LPR = lanes per row = D / 8 (each lane holds 8 bf16 = 16 bytes of a row). A lane group is
 // 2*LPR lanes: the first LPR stream the K row of a position, the other LPR its V row, so both
 // halves see the same bucket boundaries (for D = 128 a group is exactly one warp: no divergence).
-// grid.x = units * slices. Dynamic shared memory: the unit's C anchors.
+// grid.x = units * slices (equal slices of at most 256 rows). Dynamic shared memory: the unit's C anchors.
 template <int LPR>
 __global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int32_t *__restrict__ anchor_pos,
@@ -71,7 +71,8 @@ merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int
     for (int k = threadIdx.x; k < C; k += kMergeThreads) anch[k] = ap[k];
     __syncthreads();
 
-    const int R0 = slice * kRowsPerCta, R1 = min(R0 + kRowsPerCta, T);
+    const int slice_rows = (T + slices - 1) / slices;      // equal slices: at most kRowsPerCta rows each
+    const int R0 = slice * slice_rows, R1 = min(R0 + slice_rows, T);
     const int part = (R1 - R0 + G - 1) / G;
     const int ra = min(R0 + g * part, R1), rb = min(ra + part, R1);
     int k = first_bucket_from(anch, C, ra);
