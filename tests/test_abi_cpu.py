@@ -106,3 +106,62 @@ def test_ratio_cache_init_validation(L):
     assert f(C.byref(c), p, p, 1, 2, 64, 64, 6, 8, 0.5, 40, ring) == 4        # fewer rows than the offset
     assert f(C.byref(c), p, p, 1, 2, 64, 64, 20, 8, 0.0, 40, ring) == 4       # ratio out of range
     assert f(C.byref(c), p, p, 1, 2, 64, 64, 20, 8, 0.5, 10, ring) == 4       # fewer tokens seen than rows held
+
+
+def test_statistic_prefix_and_from_lse_reject_bad_arguments_on_the_host(L):
+    p = 0x10000
+    ws = 1 << 20
+    f = L.ec_importance_statistic
+    assert f(p, None, p, None, 1, 1, 16, 0, 64, 1.0, 0, 0.0, p, ws, None) == 1            # NULL
+    assert f(p, p, p, None, 1, 1, 0, 4, 64, 1.0, 0, 0.0, p, ws, None) == 2                # no query
+    assert f(p, p, p, None, 1, 1, 16, -1, 64, 1.0, 0, 0.0, p, ws, None) == 2              # negative prefix
+    assert f(p, p, p, None, 1, 1, 16, 16384, 64, 1.0, 0, 0.0, p, ws, None) == 2           # P + Tq too long
+    assert f(p, p, p, None, 1, 1, 16, 0, 64, 1.0, 4, 0.0, p, ws, None) == 4               # unknown statistic
+    assert f(p, p, p, None, 1, 1, 16, 0, 64, 1.0, 3, 0.0, p, ws, None) == 4               # beta outside (0, 1)
+    assert f(p, p, p, None, 1, 1, 16, 0, 64, 1.0, 3, 1.0, p, ws, None) == 4
+    assert f(p, p, p, p + 4, 1, 1, 16, 0, 64, 1.0, 1, 0.0, p, ws, None) == 3              # lse alignment
+    assert f(p, p, p, None, 1, 1, 16, 0, 64, 1.0, 2, 0.0, p, 8, None) == 5                # workspace too small
+    g = L.ec_importance_prefix
+    assert g(p, p, None, None, 1, 1, 16, 3, 64, 1.0, p, ws, None) == 1
+    assert g(p, p, p, None, 1, 1, 16, 3, 64, float("nan"), p, ws, None) == 4
+    h = L.ec_importance_from_lse
+    assert h(p, p, None, p, 1, 1, 16, 64, 1.0, p, ws, None) == 1                          # lse missing
+    assert h(p, p, p, p, 1, 1, 16, 32, 1.0, p, ws, None) == 2
+
+
+def test_cache_concat_rejects_bad_arguments_on_the_host(L):
+    p = 0x10000
+    c = ec.ec_cache()
+    assert L.ec_cache_init(C.byref(c), p, p, 2, 3, 64, 16, 8, 8, 4) == 0
+    f = L.ec_cache_concat
+    assert f(C.byref(c), None, p, 4, p, p, None) == 1
+    assert f(None, p, p, 4, p, p, None) == 1
+    assert f(C.byref(c), p, p, 0, p, p, None) == 4                                        # no new rows
+    assert f(C.byref(c), p, p + 2, 4, p, p, None) == 3
+    c.ring_head = 4                                                                       # outside 0..offset-1
+    assert f(C.byref(c), p, p, 4, p, p, None) == 4
+    c.ring_head = 0
+    c.len = 0                                                                             # nothing cached yet
+    assert f(C.byref(c), p, p, 4, p, p, None) == 4
+    ring = (C.c_int * 4)()
+    r = ec.ec_cache()
+    assert L.ec_cache_init_ratio(C.byref(r), p, p, 1, 2, 64, 64, 20, 4, 0.5, 40, ring) == 0
+    assert f(C.byref(r), p, p, 4, p, p, None) == 4                                        # queue order not tracked
+
+
+def test_select_compact_and_noalloc_validation(L):
+    p = 0x10000
+    ws = 1 << 20
+    f = L.ec_select_compact
+    assert f(p, p, p, 2, 4, 16, 64, 8, 3, 0, 0, p, p, 8, p, None, p, ws, None) == 4       # 8 units not a multiple of 3
+    assert f(p, p, p, 2, 4, 16, 64, 8, 0, 0, 0, p, p, 8, p, None, p, ws, None) == 4       # share < 1
+    assert f(p, p, p, 2, 4, 16, 64, 8, 4, 0, 2, p, p, 8, p, None, p, ws, None) == 4       # unknown compaction
+    assert L.ec_select_compact_workspace(2, 4, 16, 64, 8, 4) >= 256 + 2 * 16 * 4
+    assert L.ec_select_compact_workspace(2, 4, 16, 64, 8, 3) == 0
+    assert L.ec_decode_noalloc_capacity() == 2 << 20
+    big = ec.ec_cache()
+    assert L.ec_cache_init(C.byref(big), p, p, 1024, 64, 128, 128, 128, 128, 16) == 0     # 65536 units
+    assert L.ec_decode_workspace(C.byref(big)) > L.ec_decode_noalloc_capacity()
+    ev = C.c_int(0)
+    assert L.ec_decode_step_noalloc(p, p, p, C.byref(big), 1.0, p, C.byref(ev), None, None) == 8
+    assert (big.len, big.step) == (128, 0)
