@@ -38,7 +38,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one decode_kernel launch from the ncu capture summarised in
 # profiles/decode_kernel_llava7b_b1_ncu.md, keyed by workload; valid only for the kernel source it was
 # taken on (sha1 prefix of csrc/ec_decode.cu), otherwise reported as null.
-DECODE_TRAFFIC = {"source_sha1": "ac8fbbb5c83f", "llava7b_b1": 172.17e6}
+DECODE_TRAFFIC = {"source_sha1": "98cd38b0b32c", "llava7b_b1": 172.13e6}
 
 
 def decode_traffic(workload: str):
@@ -392,9 +392,7 @@ def run_ours(args, w: wl.Workload):
     imp_flops = 2.0 * D * T * (T + 1) * units   # two passes, each 2*D flops for T(T+1)/2 causal scores
     imp_tflops = imp_flops / (imp_ms * 1e-3) / 1e12
     # kernels per pass: two importance passes, selection, merge, and one decode kernel per token
-    # (plus one combine kernel per token when a unit's rows are split over several CTAs)
-    splits = max(1, min(-(-148 * 4 // units), -(-(C + 1) // 64)))
-    launches_per_pass = 2 + 2 + S * (1 if splits == 1 else 2)
+    launches_per_pass = 2 + 2 + S
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

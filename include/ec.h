@@ -374,9 +374,10 @@ int ec_cache_concat(const ec_cache *c, const void *K_new_dev, const void *V_new_
  *  - The first call on each device looks up the array's device address (a one-time runtime
  *    query, made with that device current). Make that first call outside any stream capture.
  *  - All calls on a device share the one array, which keeps whatever the previous call left
- *    there. Each launch rewrites the part it reads, so no clearing is needed, but two calls
- *    whose kernels may run at the same time (different streams, different caches) race on
- *    it: serialise them.
+ *    there. Every call clears the per-unit arrival counters at the head of the array before
+ *    its kernel (a memset node on `stream`, not an allocation) and rewrites the partial
+ *    results it reads, so the caller clears nothing; but two calls whose kernels may run at
+ *    the same time (different streams, different caches) race on the array: serialise them.
  */
 size_t ec_decode_noalloc_capacity(void);
 int ec_decode_step_noalloc(const void *q_dev, const void *k_new_dev, const void *v_new_dev,

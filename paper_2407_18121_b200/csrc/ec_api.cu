@@ -247,18 +247,22 @@ size_t ec_decode_workspace(const ec_cache *c)
     if (!c) return 0;
     const int units = c->N * c->H;
     const int splits = ec::decode_splits(units, c->cap + 1);
-    return 256 + round256((size_t)units * splits * (c->D + 2) * sizeof(float));
+    // arrival counters (one int per unit) followed by the per-split partial results
+    return round256((size_t)units * sizeof(int)) + round256((size_t)units * splits * (c->D + 2) * sizeof(float));
 }
 
 }  // extern "C"
 
 namespace {
 
-// One decode step. `prev_slot` >= 0 promises that the kernel enqueued on `stream` right before
+// One decode step. `fresh_ws`: nothing is known about the workspace's contents, so the arrival
+// counters are cleared first (later steps of a native loop find them cleared by the kernel).
+// `prev_slot` >= 0 promises that the kernel enqueued on `stream` right before
 // this call is the decode step that stored cache row `prev_slot` and nothing else this step
 // reads; the kernel may then read the rest of the cache while that step is still finishing.
 int decode_step_impl(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
-                     int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream, int prev_slot)
+                     int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream, int prev_slot,
+                     bool fresh_ws)
 {
     if (!q || !k_new || !v_new || !c || !out || !evicted_slot) return EC_ERR_NULL;
     if (!c->Kc || !c->Vc) return EC_ERR_NULL;
@@ -301,9 +305,16 @@ int decode_step_impl(const void *q, const void *k_new, const void *v_new, ec_cac
     }
     const int units = c->N * c->H;
     const int splits = ec::decode_splits(units, c->len + 1);
-    float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
-    cudaError_t e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, prev_slot,
-                                      scale, out, partials, splits, (cudaStream_t)stream);
+    const size_t counter_bytes = round256((size_t)units * sizeof(int));
+    int *counters = static_cast<int *>(ws);
+    float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + counter_bytes);
+    cudaError_t e;
+    if (fresh_ws && ec::decode_splits(units, c->cap + 1) > 1) {
+        e = cudaMemsetAsync(counters, 0, (size_t)units * sizeof(int), (cudaStream_t)stream);
+        if (e != cudaSuccess) return EC_ERR_CUDA;
+    }
+    e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, prev_slot, scale, out,
+                          partials, counters, splits, (cudaStream_t)stream);
     if (e != cudaSuccess) return EC_ERR_CUDA;
     if (ratio) {
         // the new row is now the newest; the ring's oldest entry either left or stops being tracked
@@ -329,7 +340,7 @@ extern "C" {
 int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
                    int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream)
 {
-    return decode_step_impl(q, k_new, v_new, c, scale, out, evicted_slot, slot_written, ws, ws_bytes, stream, -1);
+    return decode_step_impl(q, k_new, v_new, c, scale, out, evicted_slot, slot_written, ws, ws_bytes, stream, -1, true);
 }
 
 int ec_decode_steps(const void *q, const void *k_new, const void *v_new, int steps, ec_cache *c, float scale,
@@ -343,7 +354,7 @@ int ec_decode_steps(const void *q, const void *k_new, const void *v_new, int ste
         int ev = -1, slot = -1;
         int st = decode_step_impl(static_cast<const char *>(q) + s * stride, static_cast<const char *>(k_new) + s * stride,
                                   static_cast<const char *>(v_new) + s * stride, c, scale,
-                                  static_cast<char *>(out) + s * stride, &ev, &slot, ws, ws_bytes, stream, prev);
+                                  static_cast<char *>(out) + s * stride, &ev, &slot, ws, ws_bytes, stream, prev, s == 0);
         if (st != EC_OK) return st;
         if (evicted_slots) evicted_slots[s] = ev;
         prev = slot;

@@ -76,8 +76,9 @@ cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos
                          int n_keep, void *Kc, void *Vc, int cap, cudaStream_t stream);
 
 int decode_splits(int units, int rows);
+// splits > 1: `counters` (units ints) must be zero when the launch starts; the kernel leaves them zero.
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
                           int units, int D, int cap, int len, int write_slot, int defer_row, float scale, void *out,
-                          float *partials, int splits, cudaStream_t stream);
+                          float *partials, int *counters, int splits, cudaStream_t stream);
 
 }  // namespace ec

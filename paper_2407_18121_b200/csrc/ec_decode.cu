@@ -23,6 +23,10 @@ namespace {
 #define EC_DEC_MIN_CTAS 8
 #endif
 constexpr int kDecThreads = EC_DEC_THREADS;
+#ifndef EC_DEC_TARGET
+#define EC_DEC_TARGET (148 * 4)
+#endif
+constexpr int kMaxSplits = EC_DEC_TARGET;     // CTAs aimed at when there are fewer units than that; also the most splits a unit gets
 constexpr int kBlk = 8;                       // rows per block of a lane group
 
 // The cache is written later in the same kernel, so no read-only (.nc) path here.
@@ -136,17 +140,21 @@ __device__ __forceinline__ void process_block(GroupState &st, const float2 (&q2)
 
 // grid.x = units * splits. Rows 0..len-1 come from the cache, row `len` is the new token.
 // splits == 1: writes out (bf16) and stores the new row into `write_slot`.
-// splits  > 1: writes (acc[D], max, sum) per split to `partials`; the combine kernel finishes.
+// splits  > 1: every CTA writes (acc[D], max, sum) of its rows to `partials` and counts itself in
+// `counters[unit]`; the CTA that arrives last (nobody waits for anybody) merges the unit's partials,
+// writes out, stores the new row and puts the counter back to zero for the next launch.
 template <int LPR>
 __global__ void __launch_bounds__(kDecThreads, EC_DEC_MIN_CTAS)
 decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
               uint4 *Kc, uint4 *Vc, int cap, int len, int write_slot, int defer_row, float scale_log2e,
-              __nv_bfloat16 *__restrict__ out, float *__restrict__ partials, int splits)
+              __nv_bfloat16 *__restrict__ out, float *partials, int *counters, int splits)
 {
     constexpr int D = LPR * 8;
     constexpr int G = kDecThreads / LPR;
     __shared__ float sm_acc[G][D];
     __shared__ float sm_m[G], sm_l[G];
+    __shared__ int sm_last;
+    __shared__ float sm_pm[kMaxSplits], sm_pl[kMaxSplits];   // (max, sum) of every split of the unit
 
     // Launched with programmatic stream serialization. defer_row < 0: nothing in global memory
     // is touched before the previous kernel of the stream has completed. defer_row >= 0: the
@@ -257,42 +265,48 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
             if (d == 0) { p[D] = M; p[D + 1] = L; }
         }
     }
-    if (splits == 1 && threadIdx.x >= kDecThreads - 2 * LPR) {
+    bool finish = splits == 1;
+    if (splits > 1) {
+        // last arriver of the unit: its own partial and, through the fences, everybody else's are visible
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) sm_last = (atomicAdd(counters + unit, 1) == splits - 1);
+        __syncthreads();
+        finish = sm_last != 0;
+        if (finish) {
+            __threadfence();
+            if (threadIdx.x == 0) counters[unit] = 0;
+            // the splits' (max, sum) pairs first, all loads in flight at once, then their weights
+            const float *p = partials + (size_t)unit * splits * (D + 2);
+            for (int sp = threadIdx.x; sp < splits; sp += kDecThreads) {
+                sm_pm[sp] = __ldcg(p + (size_t)sp * (D + 2) + D);
+                sm_pl[sp] = __ldcg(p + (size_t)sp * (D + 2) + D + 1);
+            }
+            __syncthreads();
+            float M = -INFINITY;
+            for (int sp = 0; sp < splits; ++sp) M = fmaxf(M, sm_pm[sp]);
+            float L = 0.f;
+            for (int sp = 0; sp < splits; ++sp) {
+                const float ms = sm_pm[sp];
+                L = fmaf(sm_pl[sp], (ms == -INFINITY) ? 0.f : fast_exp2(ms - M), L);
+            }
+            const float inv_l = 1.f / L;
+            for (int d = threadIdx.x; d < D; d += kDecThreads) {
+                float A = 0.f;
+#pragma unroll 4
+                for (int sp = 0; sp < splits; ++sp) {
+                    const float ms = sm_pm[sp];
+                    A = fmaf(__ldcg(p + (size_t)sp * (D + 2) + d), (ms == -INFINITY) ? 0.f : fast_exp2(ms - M), A);
+                }
+                out[(size_t)unit * D + d] = __float2bfloat16_rn(A * inv_l);
+            }
+        }
+    }
+    // the new row takes the freed slot once every CTA of the unit has read its rows
+    if (finish && threadIdx.x >= kDecThreads - 2 * LPR) {
         const int i = threadIdx.x - (kDecThreads - 2 * LPR);
         if (i < LPR) Kcu[(size_t)write_slot * LPR + i] = knu[i];
         else         Vcu[(size_t)write_slot * LPR + (i - LPR)] = vnu[i - LPR];
-    }
-}
-
-// Merges the per-split partials of one unit, writes out and stores the new row.
-template <int LPR>
-__global__ void combine_kernel(const float *__restrict__ partials, int splits,
-                               const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-                               uint4 *Kc, uint4 *Vc, int cap, int write_slot, __nv_bfloat16 *__restrict__ out)
-{
-    constexpr int D = LPR * 8;
-    grid_dependency_wait();
-    grid_launch_dependents();
-    const int unit = blockIdx.x;
-    const int d = threadIdx.x;
-    const float *p = partials + (size_t)unit * splits * (D + 2);
-    if (d < D) {
-        float M = -INFINITY;
-        for (int s = 0; s < splits; ++s) M = fmaxf(M, p[(size_t)s * (D + 2) + D]);
-        float L = 0.f, A = 0.f;
-        for (int s = 0; s < splits; ++s) {
-            const float ms = p[(size_t)s * (D + 2) + D];
-            const float w = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
-            L = fmaf(p[(size_t)s * (D + 2) + D + 1], w, L);
-            A = fmaf(p[(size_t)s * (D + 2) + d], w, A);
-        }
-        out[(size_t)unit * D + d] = __float2bfloat16_rn(A / L);
-    }
-    if (d < 2 * LPR) {
-        uint4 *Kcu = Kc + (size_t)unit * cap * LPR;
-        uint4 *Vcu = Vc + (size_t)unit * cap * LPR;
-        if (d < LPR) Kcu[(size_t)write_slot * LPR + d] = k_new[(size_t)unit * LPR + d];
-        else         Vcu[(size_t)write_slot * LPR + (d - LPR)] = v_new[(size_t)unit * LPR + (d - LPR)];
     }
 }
 
@@ -302,7 +316,7 @@ __global__ void combine_kernel(const float *__restrict__ partials, int splits,
 // the GPU; every split keeps at least 64 rows.
 int decode_splits(int units, int rows)
 {
-    const int target = 148 * 4;
+    const int target = kMaxSplits;
     int s = (target + units - 1) / units;
     int max_s = (rows + 63) / 64;
     if (s > max_s) s = max_s;
@@ -331,27 +345,24 @@ cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, unsigned 
 template <int LPR>
 cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc, int units,
                             int cap, int len, int write_slot, int defer_row, float sl2, void *out, float *partials,
-                            int splits, cudaStream_t stream)
+                            int *counters, int splits, cudaStream_t stream)
 {
-    cudaError_t e = launch_overlapped(decode_kernel<LPR>, (unsigned)(units * splits), (unsigned)kDecThreads, stream,
-                                      (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc,
-                                      (uint4 *)Vc, cap, len, write_slot, splits == 1 ? defer_row : -1, sl2, (__nv_bfloat16 *)out,
-                                      partials, splits);
-    if (e != cudaSuccess || splits == 1) return e;
-    return launch_overlapped(combine_kernel<LPR>, (unsigned)units, (unsigned)(LPR * 8), stream,
-                             (const float *)partials, splits, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc,
-                             (uint4 *)Vc, cap, write_slot, (__nv_bfloat16 *)out);
+    return launch_overlapped(decode_kernel<LPR>, (unsigned)(units * splits), (unsigned)kDecThreads, stream,
+                             (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap, len,
+                             write_slot, defer_row, sl2, (__nv_bfloat16 *)out, partials, counters, splits);
 }
 
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
                           int units, int D, int cap, int len, int write_slot, int defer_row, float scale, void *out,
-                          float *partials, int splits, cudaStream_t stream)
+                          float *partials, int *counters, int splits, cudaStream_t stream)
 {
     const float sl2 = scale * 1.4426950408889634f;
     if ((long long)units * splits > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     if (D == 128)
-        return launch_decode_t<16>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials, splits, stream);
-    return launch_decode_t<8>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials, splits, stream);
+        return launch_decode_t<16>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials,
+                                   counters, splits, stream);
+    return launch_decode_t<8>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials, counters,
+                              splits, stream);
 }
 
 }  // namespace ec

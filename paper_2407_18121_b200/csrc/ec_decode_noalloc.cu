@@ -1,7 +1,7 @@
 // ec_decode_step_noalloc: the decode step for callers that cannot allocate device memory.
 //
-// The ordinary ec_decode_step needs a caller-provided workspace (the per-split partial
-// results that the combine kernel merges). Some hosts cannot provide one: an inference
+// The ordinary ec_decode_step needs a caller-provided workspace (per-unit arrival counters
+// and the per-split partial results that the last CTA of a unit merges). Some hosts cannot provide one: an inference
 // server that hands all of the GPU's memory to its own pool at start-up and forbids
 // cudaMalloc afterwards, a plug-in whose execute callback may not allocate, or a latency-
 // critical loop that cannot afford cudaMalloc's implicit device synchronisation. For them
@@ -52,8 +52,9 @@ int ec_decode_step_noalloc(const void *q, const void *k_new, const void *v_new, 
     void *scratch = nullptr;
     int st = scratch_address(&scratch);
     if (st != EC_OK) return st;
-    // Partial results are fully rewritten by every launch before the combine kernel reads
-    // them, so nothing in the array has to start at zero.
+    // What has to start at zero (the arrival counters at the head of the array) is cleared by
+    // ec_decode_step itself with a memset node before its kernel; the partial results are
+    // rewritten by every launch before they are read.
     return ec_decode_step(q, k_new, v_new, c, scale, out, evicted_slot, slot_written, scratch, kNoAllocBytes, stream);
 }
 

@@ -303,6 +303,39 @@ def test_decode_steps_native_loop_matches_single_steps():
     assert (cb.len, cb.ring_head, cb.step) == (C, S % d, S)
 
 
+@pytest.mark.parametrize("N,H,D,C,len0,offset,steps", [
+    (1, 8, 128, 200, 40, 16, 190),      # grows from one CTA per unit to four, then evicts at the budget
+    (1, 3, 64, 700, 700, 25, 30),       # eleven CTAs per unit from the first step on
+    (4, 32, 128, 192, 192, 16, 24),     # 128 units: five CTAs each, consecutive steps overlap
+])
+def test_split_units_with_a_dirty_workspace(N, H, D, C, len0, offset, steps):
+    """Few units: a unit's rows are shared by several CTAs and the last one to arrive merges their
+    partial results. The workspace starts full of ones (arrival counters included), is reused by
+    single-step calls and by the native loop, and the outputs must match the oracle throughout."""
+    rng = np.random.default_rng(len0 + steps)
+    scale = 1.0 / math.sqrt(D)
+    K0b, V0b = rand_bits(rng, (N, H, len0, D)), rand_bits(rng, (N, H, len0, D))
+    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=C + 1)
+    Kc = torch.zeros((N, H, C, D), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    Kc[:, :, :len0], Vc[:, :, :len0] = dev_bf16(K0b), dev_bf16(V0b)
+    cache = ec.ec_cache_init(Kc, Vc, len0, C, offset)
+    ws = torch.full((ec.ec_decode_workspace(cache),), 0xFF, dtype=torch.uint8, device="cuda")
+    qb, kb, vb = (rand_bits(rng, (steps, N, H, D)) for _ in range(3))
+    want = np.stack([queue.step(qb[s], kb[s], vb[s], scale, policy=orc.POLICY_FIXED, budget=C, offset=offset)[0]
+                     for s in range(steps)])
+    q, k, v = dev_bf16(qb), dev_bf16(kb), dev_bf16(vb)
+    out = torch.empty((steps, N, H, D), dtype=torch.bfloat16, device="cuda")
+    single = steps // 3                                       # first third: one call per step
+    for s in range(single):
+        ec.ec_decode_step(q[s], k[s], v[s], cache, scale, out[s], ws)
+    ws.fill_(0xFF)                                            # dirty again before the native loop
+    ec.ec_decode_steps(q[single:], k[single:], v[single:], cache, scale, out[single:], ws)
+    assert cache.len == queue.len and cache.step == steps
+    for s in range(steps):
+        assert_bf16_close(out[s], want[s], f"split decode, step {s}")
+
+
 # ---------------------------------------------------------------- the whole path
 
 @pytest.mark.parametrize("name,population", [("tiny", ec.EC_PER_HEAD), ("tiny", ec.EC_LAYER_SHARED),
