@@ -251,7 +251,8 @@ def run_decode_case(N, H, D, C, cap, len0, offset, steps, scale, seed, sigma_k=1
 
 
 @pytest.mark.parametrize("N,H,D,C,offset,steps", [
-    (1, 8, 64, 128, 16, 40),        # few units: the rows of a unit are split over several CTAs
+    (1, 8, 64, 128, 16, 40),        # few units, short cache: one CTA per unit
+    (1, 8, 64, 600, 16, 12),        # few units, longer cache: the rows of a unit are split over three CTAs
     (1, 2, 128, 70, 25, 60),        # the paper's recent distance of 25
     (20, 32, 128, 96, 16, 20),      # many units: one CTA per unit
     (3, 5, 64, 33, 1, 5),           # offset 1: only the newest row is protected
@@ -304,9 +305,9 @@ def test_decode_steps_native_loop_matches_single_steps():
 
 
 @pytest.mark.parametrize("N,H,D,C,len0,offset,steps", [
-    (1, 8, 128, 200, 40, 16, 190),      # grows from one CTA per unit to four, then evicts at the budget
-    (1, 3, 64, 700, 700, 25, 30),       # eleven CTAs per unit from the first step on
-    (4, 32, 128, 192, 192, 16, 24),     # 128 units: five CTAs each, consecutive steps overlap
+    (1, 8, 128, 600, 200, 16, 420),     # grows from one CTA per unit to three, then evicts at the budget
+    (1, 3, 64, 700, 700, 25, 30),       # three CTAs per unit from the first step on
+    (4, 32, 128, 512, 512, 16, 24),     # 128 units: three CTAs each, consecutive steps overlap
 ])
 def test_split_units_with_a_dirty_workspace(N, H, D, C, len0, offset, steps):
     """Few units: a unit's rows are shared by several CTAs and the last one to arrive merges their
