@@ -165,3 +165,17 @@ def test_select_compact_and_noalloc_validation(L):
     ev = C.c_int(0)
     assert L.ec_decode_step_noalloc(p, p, p, C.byref(big), 1.0, p, C.byref(ev), None, None) == 8
     assert (big.len, big.step) == (128, 0)
+
+
+def test_header_is_plain_c(tmp_path):
+    """ec.h is a C header: a C99 translation unit that includes nothing else compiles against it
+    and can name every declared function with its declared type."""
+    import subprocess
+    names = _declared()
+    src = tmp_path / "use_ec.c"
+    body = "\n".join(f"    (void)&{n};" for n in names)
+    src.write_text('#include "ec.h"\nint main(void)\n{\n    ec_cache c;\n    (void)sizeof(c);\n' + body +
+                   "\n    return EC_OK;\n}\n")
+    r = subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-fsyntax-only",
+                        "-I", os.path.join(ROOT, "include"), str(src)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
