@@ -38,7 +38,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one decode_kernel launch (a later step of the loop) from the ncu capture summarised in
 # profiles/decode_kernel_llava7b_b1_ncu.md, keyed by workload; valid only for the kernel source it was
 # taken on (sha1 prefix of csrc/ec_decode.cu), otherwise reported as null.
-DECODE_TRAFFIC = {"source_sha1": "2e29faa11088", "llava7b_b1": 172.25e6}
+DECODE_TRAFFIC = {"source_sha1": "00c4a558985a", "llava7b_b1": 172.6e6}
 
 
 def decode_traffic(workload: str):

@@ -293,9 +293,11 @@ int ec_decode_step(const void *q_dev, const void *k_new_dev, const void *v_new_d
  * `steps` consecutive ec_decode_step calls issued from native code. Step s reads
  * q/k_new/v_new at element offset s*N*H*D of the three [steps, N, H, D] arrays and writes
  * out at the same offset. evicted_slots_host (may be NULL) receives `steps` ints.
- * All inputs of all steps must be complete on `stream` before the call: when every unit has a
- * CTA of its own, a step starts reading the cache while the previous one is still finishing
- * (only the row that step stores is read late).
+ * All inputs of all steps must be complete on `stream` before the call: from the second step
+ * on, a step starts reading its q/k_new/v_new and the cache rows that no step of the call
+ * writes (everything but the slots of the `offset` most recent rows and the rows appended
+ * during the call) while earlier steps of the call are still running; only those few rows, and
+ * every write, wait for the step before.
  */
 int ec_decode_steps(const void *q_dev, const void *k_new_dev, const void *v_new_dev, int steps,
                     ec_cache *c, float scale, void *out_dev, int *evicted_slots_host,

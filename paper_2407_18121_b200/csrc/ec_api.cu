@@ -257,11 +257,11 @@ namespace {
 
 // One decode step. `fresh_ws`: nothing is known about the workspace's contents, so the arrival
 // counters are cleared first (later steps of a native loop find them cleared by the kernel).
-// `prev_slot` >= 0 promises that the kernel enqueued on `stream` right before
-// this call is the decode step that stored cache row `prev_slot` and nothing else this step
-// reads; the kernel may then read the rest of the cache while that step is still finishing.
+// `stable_rows` >= 0 promises that the kernels enqueued on `stream` since the last full
+// dependency are decode steps of this cache which write no row below `stable_rows`; the kernel
+// may then read those rows while the earlier steps are still running.
 int decode_step_impl(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
-                     int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream, int prev_slot,
+                     int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream, int stable_rows,
                      bool fresh_ws)
 {
     if (!q || !k_new || !v_new || !c || !out || !evicted_slot) return EC_ERR_NULL;
@@ -313,7 +313,7 @@ int decode_step_impl(const void *q, const void *k_new, const void *v_new, ec_cac
         e = cudaMemsetAsync(counters, 0, (size_t)units * sizeof(int), (cudaStream_t)stream);
         if (e != cudaSuccess) return EC_ERR_CUDA;
     }
-    e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, prev_slot, scale, out,
+    e = ec::launch_decode(q, k_new, v_new, c->Kc, c->Vc, units, c->D, c->cap, c->len, slot, stable_rows, scale, out,
                           partials, counters, splits, (cudaStream_t)stream);
     if (e != cudaSuccess) return EC_ERR_CUDA;
     if (ratio) {
@@ -349,15 +349,25 @@ int ec_decode_steps(const void *q, const void *k_new, const void *v_new, int ste
     if (steps < 0) return EC_ERR_ARG;
     if (!c) return EC_ERR_NULL;
     const size_t stride = (size_t)c->N * c->H * c->D * 2;   // bytes of one [N, H, D] bf16 step
-    int prev = -1;       // the first step of the call knows nothing about the kernel before it
+    // Rows no step of this call will write: new rows go to the slots of the `offset` most recent
+    // rows (the ring of a full fixed-budget cache, the tracked recent slots of the ratio policy) or
+    // are appended at len and beyond. The first step knows nothing about the kernel before it.
+    int stable = c->len;
+    if (c->policy == EC_POLICY_RATIO) {
+        if (c->recent_slots_host && c->offset >= 1)
+            for (int i = 0; i < c->offset; ++i) stable = stable < c->recent_slots_host[i] ? stable : c->recent_slots_host[i];
+    } else if (c->budget - c->offset < stable) {
+        stable = c->budget - c->offset;
+    }
+    if (stable < 0) stable = 0;
     for (int s = 0; s < steps; ++s) {
         int ev = -1, slot = -1;
         int st = decode_step_impl(static_cast<const char *>(q) + s * stride, static_cast<const char *>(k_new) + s * stride,
                                   static_cast<const char *>(v_new) + s * stride, c, scale,
-                                  static_cast<char *>(out) + s * stride, &ev, &slot, ws, ws_bytes, stream, prev, s == 0);
+                                  static_cast<char *>(out) + s * stride, &ev, &slot, ws, ws_bytes, stream,
+                                  s == 0 ? -1 : stable, s == 0);
         if (st != EC_OK) return st;
         if (evicted_slots) evicted_slots[s] = ev;
-        prev = slot;
     }
     return EC_OK;
 }

@@ -77,8 +77,9 @@ cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos
 
 int decode_splits(int units, int rows);
 // splits > 1: `counters` (units ints) must be zero when the launch starts; the kernel leaves them zero.
+// defer_from >= 0: the kernels in front on `stream` are decode steps that write no cache row below defer_from.
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
-                          int units, int D, int cap, int len, int write_slot, int defer_row, float scale, void *out,
+                          int units, int D, int cap, int len, int write_slot, int defer_from, float scale, void *out,
                           float *partials, int *counters, int splits, cudaStream_t stream);
 
 }  // namespace ec

@@ -147,8 +147,8 @@ __device__ __forceinline__ void process_block(GroupState &st, const float2 (&q2)
 template <int LPR>
 __global__ void __launch_bounds__(kDecThreads, EC_DEC_MIN_CTAS)
 decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-              uint4 *Kc, uint4 *Vc, int cap, int len, int write_slot, int defer_row, float scale_log2e,
-              __nv_bfloat16 *__restrict__ out, float *partials, int *counters, int splits)
+              uint4 *Kc, uint4 *Vc, int cap, int len, int write_slot, int defer_from, float scale_log2e,
+              __nv_bfloat16 *__restrict__ out, float *partials, int *counters, int splits, int release_early)
 {
     constexpr int D = LPR * 8;
     constexpr int G = kDecThreads / LPR;
@@ -157,16 +157,16 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
     __shared__ int sm_last;
     __shared__ float sm_pm[kMaxSplits], sm_pl[kMaxSplits];   // (max, sum) of every split of the unit
 
-    // Launched with programmatic stream serialization. defer_row < 0: nothing in global memory
-    // is touched before the previous kernel of the stream has completed. defer_row >= 0: the
-    // previous kernel is the decode step before this one, which changes nothing this step reads
-    // except cache row `defer_row` (the row it stored); everything else is read first, and only
-    // the block holding that row, and every write, wait for the predecessor. The next launch is
-    // released only after that wait, so at most two consecutive steps ever overlap.
-    if (defer_row < 0) {
-        grid_dependency_wait();
-        grid_launch_dependents();
-    }
+    // Launched with programmatic stream serialization. defer_from < 0: nothing in global memory
+    // is touched before the previous kernel of the stream has completed. defer_from >= 0: the
+    // kernels in front are earlier decode steps of the same call, and none of them writes a cache
+    // row below `defer_from` (new rows only ever go to the slots of the most recent rows or are
+    // appended). Those stable rows are read at once, however many earlier steps are still in
+    // flight, and the next step is released before anything else, so that its launch latency and
+    // its reading hide behind this step; the rows from `defer_from` on, and every write, wait for
+    // the predecessor to complete (and with it all steps before it).
+    if (defer_from < 0) grid_dependency_wait();
+    if (defer_from < 0 || release_early) grid_launch_dependents();
 
     const int unit = blockIdx.x / splits;
     const int split = blockIdx.x - unit * splits;
@@ -202,18 +202,18 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
 
     const uint4 *Kl = Kcu + l, *Vl = Vcu + l;
     const bool has_tail = r0 + nfull * kBlk < r1;
-    const int bd = (defer_row >= r0 && defer_row < r1) ? (defer_row - r0) / kBlk : -1;   // block put off
-    for (int b = g; b < nfull; b += G)
-        if (b != bd) process_block<LPR, false>(st, q2, Kl, Vl, r0 + b * kBlk, r1, l, gmask);
-    if (has_tail && (nfull % G) == g && bd != nfull)
-        process_block<LPR, true>(st, q2, Kl, Vl, r0 + nfull * kBlk, r1, l, gmask);
-    if (defer_row >= 0) {
+    if (defer_from < 0) {
+        for (int b = g; b < nfull; b += G) process_block<LPR, false>(st, q2, Kl, Vl, r0 + b * kBlk, r1, l, gmask);
+        if (has_tail && (nfull % G) == g) process_block<LPR, true>(st, q2, Kl, Vl, r0 + nfull * kBlk, r1, l, gmask);
+    } else {
+        // whole blocks of stable rows first; the rest after the predecessor has completed
+        const int early = (min(max(defer_from, r0), r1) - r0) / kBlk;
+        for (int b = g; b < early; b += G) process_block<LPR, false>(st, q2, Kl, Vl, r0 + b * kBlk, r1, l, gmask);
         grid_dependency_wait();
-        grid_launch_dependents();
-        if (bd >= 0 && (bd % G) == g) {
-            if (bd < nfull) process_block<LPR, false, true>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
-            else            process_block<LPR, true, true>(st, q2, Kl, Vl, r0 + bd * kBlk, r1, l, gmask);
-        }
+        if (!release_early) grid_launch_dependents();
+        for (int b = early + (g - early % G + G) % G; b < nfull; b += G)     // block b stays with group b % G
+            process_block<LPR, false, true>(st, q2, Kl, Vl, r0 + b * kBlk, r1, l, gmask);
+        if (has_tail && (nfull % G) == g) process_block<LPR, true, true>(st, q2, Kl, Vl, r0 + nfull * kBlk, r1, l, gmask);
     }
 
     // per-lane partial sums -> group sum (rows are owned by LPR/8 lanes each)
@@ -348,24 +348,28 @@ cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, unsigned 
 
 template <int LPR>
 cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc, int units,
-                            int cap, int len, int write_slot, int defer_row, float sl2, void *out, float *partials,
+                            int cap, int len, int write_slot, int defer_from, float sl2, void *out, float *partials,
                             int *counters, int splits, cudaStream_t stream)
 {
+#ifndef EC_DEC_EARLY_MIN_MB
+#define EC_DEC_EARLY_MIN_MB 24
+#endif
+    const int release_early = (double)units * len * LPR * 32.0 >= EC_DEC_EARLY_MIN_MB * 1.0e6;   // K and V bytes of a step
     return launch_overlapped(decode_kernel<LPR>, (unsigned)(units * splits), (unsigned)kDecThreads, stream,
                              (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap, len,
-                             write_slot, defer_row, sl2, (__nv_bfloat16 *)out, partials, counters, splits);
+                             write_slot, defer_from, sl2, (__nv_bfloat16 *)out, partials, counters, splits, release_early);
 }
 
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
-                          int units, int D, int cap, int len, int write_slot, int defer_row, float scale, void *out,
+                          int units, int D, int cap, int len, int write_slot, int defer_from, float scale, void *out,
                           float *partials, int *counters, int splits, cudaStream_t stream)
 {
     const float sl2 = scale * 1.4426950408889634f;
     if ((long long)units * splits > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     if (D == 128)
-        return launch_decode_t<16>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials,
+        return launch_decode_t<16>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_from, sl2, out, partials,
                                    counters, splits, stream);
-    return launch_decode_t<8>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_row, sl2, out, partials, counters,
+    return launch_decode_t<8>(q, k_new, v_new, Kc, Vc, units, cap, len, write_slot, defer_from, sl2, out, partials, counters,
                               splits, stream);
 }
 
