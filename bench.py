@@ -278,8 +278,6 @@ def run_ours(args, w: wl.Workload):
     Q, K, V = Qh.cuda(), Kh.cuda(), Vh.cuda()
     q, k, v = qh.cuda(), kh.cuda(), vh.cuda()
     out = torch.empty_like(q)
-    out_h = torch.empty(q.shape, dtype=torch.bfloat16).pin_memory()
-    anchors_h = torch.empty((N, H, ec.ec_keep_count(T, wr.keep_ratio)), dtype=torch.int32).pin_memory()
 
     sess = ElasticCacheSession(N, H, T, D, wr.keep_ratio, wr.offset, wr.scale)
     C = sess.n_keep
@@ -354,23 +352,47 @@ def run_ours(args, w: wl.Workload):
         barrier()
         graph_ms = g0.elapsed_time(g1) / reps
 
-    # end to end: inputs start in pinned host memory, results are read back every pass
-    for _ in range(max(1, min(args.warmup, 2))):
-        sess.compress_host(Qh, Kh, Vh, anchors_h)
-        sess.decode_host(qh, kh, vh, out_h)
+    # end to end: inputs start in pinned host memory, results are read back every pass. Two passes are
+    # in flight, each with its own session, stream and host result buffers, so that the upload of the
+    # next pass's prompt overlaps the decode loop of this one (a serving loop with double buffering);
+    # every copy of every pass lies inside the timed region.
+    lanes = []
+    for _ in range(2):
+        lane_sess = ElasticCacheSession(N, H, T, D, wr.keep_ratio, wr.offset, wr.scale)
+        lanes.append((lane_sess, torch.cuda.Stream(), torch.empty(q.shape, dtype=torch.bfloat16).pin_memory(),
+                      torch.empty((N, H, C), dtype=torch.int32).pin_memory()))
+
+    def e2e_pass(i):
+        lane_sess, lane_stream, lane_out, lane_anchors = lanes[i % 2]
+        with torch.cuda.stream(lane_stream):
+            a = lane_sess.compress_host(Qh, Kh, Vh, lane_anchors)
+            b, c = lane_sess.decode_host(qh, kh, vh, lane_out)
+        return a + b, c + lane_anchors.numel() * 4
+
+    def fork():
+        for _, lane_stream, _, _ in lanes:
+            lane_stream.wait_stream(stream)
+
+    def join():
+        for _, lane_stream, _, _ in lanes:
+            stream.wait_stream(lane_stream)
+
+    fork()
+    for i in range(2):
+        e2e_pass(i)
+    join()
     barrier()
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
-    e2e_steps = max(1, min(args.steps, 3))
+    e2e_steps = max(2, min(args.steps, 6))
     e0.record(stream)
-    for _ in range(e2e_steps):
-        h2d_a = sess.compress_host(Qh, Kh, Vh, anchors_h)
-        h2d_b, d2h_b = sess.decode_host(qh, kh, vh, out_h)
+    fork()
+    for i in range(e2e_steps):
+        h2d, d2h = e2e_pass(i)
+    join()
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    h2d = h2d_a + h2d_b
-    d2h = d2h_b + anchors_h.numel() * 4
 
     ms_per_step = total_ms / args.steps
     ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms = max_over_ranks([ms_per_step, e2e_ms, dec_ms, mrg_ms, imp_ms], "cuda")
@@ -417,7 +439,8 @@ def run_ours(args, w: wl.Workload):
         "importance": {"achieved": imp_tflops, "unit": "TFLOP/s", "frac": imp_tflops / peaks["bf16_tflops"],
                        "flops_per_call": imp_flops},
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "pipeline": "two passes in flight: the next pass's prompt upload overlaps this pass's decode loop"},
         "gpu_launches": launches_per_pass * args.steps,
         "clocks": clocks,
     }
