@@ -499,13 +499,14 @@ def test_select_compact_populations_and_eviction(share_kind, compaction):
         assert_bf16_close(Vc, orc.merge(Vb, lo, hi), "merged V")
 
 
-def test_decode_steps_overlapped_loop_with_many_units():
-    """With enough units for one CTA per unit, the native loop lets step s+1 read the cache while
-    step s is still finishing, putting off only the row step s stores. Rows stored by earlier steps
-    sit in full blocks and in the ragged last block here; results must match the one-step calls
-    and the oracle."""
+@pytest.mark.parametrize("N", [20, 64])       # 15 MB per step: successor released after the wait; 47 MB: released at once
+def test_decode_steps_overlapped_loop_with_many_units(N):
+    """With enough units for one CTA per unit, the native loop lets later steps read the rows no step
+    writes (here the first 35 of 45) while earlier steps are still in flight; the ring of the 10 most
+    recent rows, which sits in a full block and in the ragged last block, is read after the wait.
+    Results must match the one-step calls and the oracle."""
     rng = np.random.default_rng(12)
-    N, H, D, C, d, S = 20, 32, 128, 45, 10, 33
+    H, D, C, d, S = 32, 128, 45, 10, 33
     K0b, V0b = rand_bits(rng, (N, H, C, D)), rand_bits(rng, (N, H, C, D))
     qb, kb, vb = (rand_bits(rng, (S, N, H, D)) for _ in range(3))
     K0, V0 = dev_bf16(K0b), dev_bf16(V0b)
@@ -523,7 +524,7 @@ def test_decode_steps_overlapped_loop_with_many_units():
     assert torch.equal(Ka, Kb_) and torch.equal(Va, Vb_)
     a, b = host_f64(out_a), host_f64(out_b)
     assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(a) + 1e-6).all()          # same result up to block order
-    for (n, h) in [(0, 0), (7, 13), (19, 31)]:
+    for (n, h) in [(0, 0), (7, 13), (N - 1, 31)]:
         queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b[n, h][None]), wl.bf16_bits_to_f64(V0b[n, h][None]), cap=C + 1)
         for s in range(S):
             want, _, _ = queue.step(qb[s, n, h][None], kb[s, n, h][None], vb[s, n, h][None], 0.09,
