@@ -361,9 +361,13 @@ void eco_merge(const uint16_t *X, int U, int T, int D, const int32_t *lo, const 
  * Steps: (i) append (k_new, v_new) at the tail with identity new_id; (ii) out =
  * softmax(scale * q K^T) V over all *len+1 rows; (iii) eviction:
  *   policy 0 (fixed budget): if the length exceeds `budget`, delete one row;
- *   policy 1 (retention ratio): del = int(length - n_tot*ratio) with n_tot the number
- *            of tokens seen so far including this one (Alg. 1's del_num with
- *            r = 1 - ratio); delete one row only when del >= 1.
+ *   policy 1 (retention ratio): Algorithm 1 is called after the forward pass, so its
+ *            seq_len is the cache length with the new row in it, and its n ("number of
+ *            tokens") counts every token processed so far, the new one included, just as
+ *            at the prompt call n = seq_len = T counts the whole prompt. With n_seen the
+ *            tokens processed before this step: del = int(length - (n_seen + 1)*ratio),
+ *            `ratio` being the retained fraction (Alg. 1's 1 - r); one row is deleted only
+ *            when del >= 1, otherwise the cache keeps the new row and grows.
  * The deleted queue position is length - 1 - offset (0-based), so `offset` rows stay
  * behind it. Rows after it move up by one, as the concatenation of the two slices does.
  * Returns the deleted queue position, or -1 when nothing was deleted. *evicted_id gets
@@ -371,7 +375,7 @@ void eco_merge(const uint16_t *X, int U, int T, int D, const int32_t *lo, const 
  */
 int eco_decode_step(double *Kl, double *Vl, int64_t *ids, int U, int cap, int D, int *len,
                     const uint16_t *q, const uint16_t *k_new, const uint16_t *v_new, double scale,
-                    int64_t new_id, int policy, int budget, int offset, double ratio, int64_t n_tot,
+                    int64_t new_id, int policy, int budget, int offset, double ratio, int64_t n_seen,
                     double *out, int64_t *evicted_id)
 {
     int L = *len;
@@ -407,7 +411,8 @@ int eco_decode_step(double *Kl, double *Vl, int64_t *ids, int U, int cap, int D,
     if (policy == 0) {
         del = (Lp > budget) ? 1 : 0;
     } else {
-        del = (int)floor((double)Lp - (double)n_tot * ratio);
+        const int64_t n = n_seen + 1;                       /* this step's token is counted */
+        del = (int)floor((double)Lp - (double)n * ratio);
         if (del < 0) del = 0;
     }
     if (del < 1) {

@@ -204,10 +204,11 @@ class DecodeQueue:
     """The cache as the paper's queue: rows in order, delete-by-position, fp64 contents.
 
     K0, V0: float64 [..., len, D] initial rows (identities 0..len-1). ``cap`` rows are
-    reserved so appended rows fit.
+    reserved so appended rows fit. ``n_seen``: tokens processed so far (the prompt length
+    right after the prompt call); the retention-ratio policy reads it, every step adds one.
     """
 
-    def __init__(self, K0: np.ndarray, V0: np.ndarray, cap: Optional[int] = None):
+    def __init__(self, K0: np.ndarray, V0: np.ndarray, cap: Optional[int] = None, n_seen: int = 0):
         K0 = np.ascontiguousarray(K0, np.float64)
         V0 = np.ascontiguousarray(V0, np.float64)
         assert K0.shape == V0.shape
@@ -223,9 +224,10 @@ class DecodeQueue:
         self.ids = np.full(self.cap, -1, np.int64)
         self.ids[:self.len] = np.arange(self.len)
         self.next_id = self.len
+        self.n_seen = int(n_seen)
 
     def step(self, q, k_new, v_new, scale: float, *, policy: int, budget: int = 0, offset: int,
-             ratio: float = 0.0, n_tot: int = 0):
+             ratio: float = 0.0):
         """One generation step. Returns (out float64 [..., D], evicted queue position or -1,
         evicted identity or -1)."""
         q, k_new, v_new = _bits(q), _bits(k_new), _bits(v_new)
@@ -235,11 +237,12 @@ class DecodeQueue:
         rc = _lib.eco_decode_step(_p(self.K, _f64p), _p(self.V, _f64p), _p(self.ids, _i64p), self.U,
                                   self.cap, self.D, C.byref(ln), _p(q, _u16p), _p(k_new, _u16p),
                                   _p(v_new, _u16p), float(scale), self.next_id, int(policy),
-                                  int(budget), int(offset), float(ratio), int(n_tot),
+                                  int(budget), int(offset), float(ratio), self.n_seen,
                                   _p(out, _f64p), _p(ev, _i64p))
         if rc == -2:
             raise RuntimeError("decode queue capacity exceeded")
         self.next_id += 1
+        self.n_seen += 1
         self.len = ln.value
         return out.reshape(self.lead + (self.D,)), rc, int(ev[0])
 

@@ -307,18 +307,57 @@ def test_below_budget_nothing_is_evicted():
     assert qd.len == 6
 
 
+def _golden_rows(name):
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)
+    return [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+
+
+def test_ratio_policy_hand_worked_traces():
+    """Two traces worked by hand from Algorithm 1's del_num line (tests/golden/retention_ratio_queue.txt):
+    which steps grow, which evict, which identity leaves and the queue after every step. They fix the
+    conventions a shared mistake could hide: the new token is counted in n, and seq_len is the length
+    after the append."""
+    rows = _golden_rows("retention_ratio_queue.txt")
+    cases = {}
+    for r in rows:
+        cases.setdefault((r[0], int(r[1]), float(r[2]), int(r[3])), []).append(
+            (int(r[4]), int(r[5]), int(r[6]), [int(x) for x in r[7:]]))
+    assert len(cases) == 2
+    rng = np.random.default_rng(15)
+    for (_, T, ratio, offset), steps in cases.items():
+        C = orc.keep_count(T, ratio)
+        assert C == len(steps[0][3]) - (1 if steps[0][1] < 0 else 0)
+        K0 = rng.standard_normal((2, C, 4))
+        qd = orc.DecodeQueue(K0, K0.copy(), cap=C + len(steps) + 1, n_seen=T)
+        for s, pos_want, id_want, ids_want in steps:
+            kb = _rand_bits(rng, (2, 4))
+            _, pos, ident = qd.step(kb, kb, kb, 1.0, policy=orc.POLICY_RATIO, offset=offset, ratio=ratio)
+            assert (pos, ident) == (pos_want, id_want), (T, ratio, s)
+            assert qd.identities().tolist() == ids_want, (T, ratio, s)
+            assert qd.n_seen == T + s + 1
+
+
+def test_keep_count_hand_worked_cases():
+    """Cases where the readings of N_I = gamma*T differ (tests/golden/keep_count_cases.txt): Algorithm 1's
+    int(T - T*gamma) removed rows is the one taken."""
+    rows = _golden_rows("keep_count_cases.txt")
+    assert len(rows) >= 6
+    for T, g, kept, other in rows:
+        assert orc.keep_count(int(T), float(g)) == int(kept) != int(other)
+
+
 def test_ratio_policy_follows_algorithm_1_count():
     # direct simulation of del_num = int(seq_len - n * ratio): one row leaves whenever it reaches 1
     rng = np.random.default_rng(14)
     T, ratio, d = 40, 0.3, 5
     C = orc.keep_count(T, ratio)
     K0 = rng.standard_normal((1, C, 4))
-    qd = orc.DecodeQueue(K0, K0.copy(), cap=C + 40)
+    qd = orc.DecodeQueue(K0, K0.copy(), cap=C + 40, n_seen=T)
     length = C
     for s in range(30):
         n_tot = T + s + 1
         kb = _rand_bits(rng, (1, 4))
-        _, pos, _ = qd.step(kb, kb, kb, 1.0, policy=orc.POLICY_RATIO, offset=d, ratio=ratio, n_tot=n_tot)
+        _, pos, _ = qd.step(kb, kb, kb, 1.0, policy=orc.POLICY_RATIO, offset=d, ratio=ratio)
         length += 1
         if int(length - n_tot * ratio) >= 1:
             assert pos == length - 1 - d

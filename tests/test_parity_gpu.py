@@ -407,7 +407,7 @@ def test_decode_ratio_policy_grows_and_evicts_like_the_oracle(T, ratio, offset, 
     C = orc.keep_count(T, ratio)
     cap = C + steps
     K0b, V0b = rand_bits(rng, (N, H, C, D)), rand_bits(rng, (N, H, C, D))
-    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=cap + 1)
+    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=cap + 1, n_seen=T)
     Kc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
     Vc = Guarded((N, H, cap, D), torch.bfloat16, fill=float("nan"))
     Kc.t[:, :, :C] = dev_bf16(K0b)
@@ -419,8 +419,7 @@ def test_decode_ratio_policy_grows_and_evicts_like_the_oracle(T, ratio, offset, 
     for s in range(steps):
         qb, kb, vb = rand_bits(rng, (N, H, D)), rand_bits(rng, (N, H, D)), rand_bits(rng, (N, H, D))
         len_before = cache.len
-        want, pos, ident = queue.step(qb, kb, vb, 0.1, policy=orc.POLICY_RATIO, offset=offset, ratio=ratio,
-                                      n_tot=T + s + 1)
+        want, pos, ident = queue.step(qb, kb, vb, 0.1, policy=orc.POLICY_RATIO, offset=offset, ratio=ratio)
         out = torch.empty((N, H, D), dtype=torch.bfloat16, device="cuda")
         ev, slot = ec.ec_decode_step(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), cache, 0.1, out, ws)
         assert_bf16_close(out, want, f"decode out, step {s}")
