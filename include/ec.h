@@ -267,6 +267,8 @@ int ec_cache_init(ec_cache *c, void *Kc_dev, void *Vc_dev, int N, int H, int D, 
 int ec_cache_init_ratio(ec_cache *c, void *Kc_dev, void *Vc_dev, int N, int H, int D, int cap,
                         int len, int offset, double keep_ratio, int64_t n_tot, int *recent_slots_host);
 
+/* Bytes of device scratch the decode calls need for this cache; depends on N, H, D and cap only.
+ * 0 when those fields are out of range (N, H, cap >= 1; D 64 or 128; N*H < 2^24) or c is NULL. */
 size_t ec_decode_workspace(const ec_cache *c);
 
 /*
@@ -282,7 +284,8 @@ size_t ec_decode_workspace(const ec_cache *c);
  *   evicted_slot_host            physical slot that was overwritten, or -1 when the cache
  *                                was below budget (host int, written before return)
  *   slot_written_host            physical slot now holding the new row (may be NULL)
- * Updates c->len, c->ring_head, c->step on success.
+ * Updates c->len, c->ring_head, c->step on success. The struct is the caller's: every call
+ * re-checks it (shape, alignment, policy fields) and returns an error instead of using a bad one.
  */
 int ec_decode_step(const void *q_dev, const void *k_new_dev, const void *v_new_dev,
                    ec_cache *c, float scale, void *out_dev,
@@ -298,6 +301,9 @@ int ec_decode_step(const void *q_dev, const void *k_new_dev, const void *v_new_d
  * writes (everything but the slots of the `offset` most recent rows and the rows appended
  * during the call) while earlier steps of the call are still running; only those few rows, and
  * every write, wait for the step before.
+ * The cache struct and the scalar arguments are checked before the first launch. A failure after
+ * that (a CUDA launch error; under the retention-ratio policy a cache with no room left to grow)
+ * ends the call at that step: the steps before it stay enqueued and c->step counts them.
  */
 int ec_decode_steps(const void *q_dev, const void *k_new_dev, const void *v_new_dev, int steps,
                     ec_cache *c, float scale, void *out_dev, int *evicted_slots_host,
@@ -331,7 +337,9 @@ int ec_compress_host(const void *Q_host, const void *K_host, const void *V_host,
  *   q_host, k_host, v_host, out_host   host bf16 [steps, N, H, D] (pinned for overlap)
  *   q_dev, k_dev, v_dev, out_dev       device staging of the same size
  *   upload_stream, download_stream     two further cudaStream_t, distinct from `stream`
- * The events the call creates are destroyed before it returns.
+ * The events the call creates are destroyed before it returns. Arguments are checked before the
+ * first copy is enqueued (ec_compress_host likewise); on a later failure c->step tells how many
+ * steps were enqueued.
  */
 int ec_decode_steps_host(const void *q_host, const void *k_host, const void *v_host, void *out_host,
                          void *q_dev, void *k_dev, void *v_dev, void *out_dev, int steps, int chunk,

@@ -23,6 +23,68 @@ int check_shape(int N, int H, int T, int D)
 
 }  // namespace
 
+namespace ec {
+
+// Host-only argument checks, shared by the device-tensor calls and the host-tensor calls (which
+// run them before their first copy, so that a rejected call has enqueued nothing).
+int check_importance_args(const void *Q, const void *K, const float *scores, const float *lse, int N, int H, int T, int D,
+                          float scale, const void *ws, size_t ws_bytes)
+{
+    if (!Q || !K || !scores) return EC_ERR_NULL;
+    int st = check_shape(N, H, T, D);
+    if (st != EC_OK) return st;
+    if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || (lse && !aligned(lse, 16))) return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    return EC_OK;
+}
+
+int check_select_compact_args(const void *K, const void *V, const float *scores, int N, int H, int T, int D, int n_keep,
+                              int share, int compaction, const void *Kc, const void *Vc, int cap,
+                              const int32_t *anchor_pos, const int32_t *bucket_len, const void *ws, size_t ws_bytes)
+{
+    if (!K || !V || !scores || !Kc || !Vc || !anchor_pos) return EC_ERR_NULL;
+    int st = check_shape(N, H, T, D);
+    if (st != EC_OK) return st;
+    if (n_keep < 1 || n_keep > T || cap < n_keep) return EC_ERR_ARG;
+    if (share < 1 || ((long long)N * H) % share != 0) return EC_ERR_ARG;
+    if (compaction != EC_COMPACT_MERGE && compaction != EC_COMPACT_EVICT) return EC_ERR_ARG;
+    if ((long long)N * H * cap >= (1LL << 31)) return EC_ERR_SHAPE;
+    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(scores, 4) ||
+        !aligned(anchor_pos, 4) || (bucket_len && !aligned(bucket_len, 4)))
+        return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < ec_select_compact_workspace(N, H, T, D, n_keep, share)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    return EC_OK;
+}
+
+// The caller owns the ec_cache struct and may have filled or restored it by hand: every call that
+// reads one repeats the checks of ec_cache_init / ec_cache_init_ratio.
+int check_cache(const ec_cache *c)
+{
+    if (!c) return EC_ERR_NULL;
+    if (!c->Kc || !c->Vc) return EC_ERR_NULL;
+    if (c->N < 1 || c->H < 1 || (c->D != 64 && c->D != 128) || c->cap < 1) return EC_ERR_SHAPE;
+    if ((long long)c->N * c->H * c->cap >= (1LL << 31) || (long long)c->N * c->H >= (1LL << 24)) return EC_ERR_SHAPE;
+    if (!aligned(c->Kc, 16) || !aligned(c->Vc, 16)) return EC_ERR_ALIGN;
+    if (c->policy == EC_POLICY_RATIO) {
+        if (!c->recent_slots_host) return EC_ERR_NULL;
+        if (c->offset < 1 || c->len < c->offset || c->len > c->cap || c->recent_head < 0 ||
+            c->recent_head >= c->offset || !(c->keep_ratio > 0.0 && c->keep_ratio <= 1.0) || c->n_tot < c->len)
+            return EC_ERR_ARG;
+    } else if (c->policy == EC_POLICY_FIXED) {
+        if (c->budget < 2 || c->budget > c->cap || c->len < 0 || c->len > c->budget || c->offset < 1 ||
+            c->offset > c->budget - 1 || c->ring_head < 0 || c->ring_head >= c->offset)
+            return EC_ERR_ARG;
+    } else {
+        return EC_ERR_ARG;
+    }
+    return EC_OK;
+}
+
+}  // namespace ec
+
 extern "C" {
 
 const char *ec_status_string(int status)
@@ -62,13 +124,8 @@ size_t ec_importance_workspace(int N, int H, int T, int D)
 int ec_importance(const void *Q, const void *K, float *scores, float *lse, int N, int H, int T, int D,
                   float scale, void *ws, size_t ws_bytes, void *stream)
 {
-    if (!Q || !K || !scores) return EC_ERR_NULL;
-    int st = check_shape(N, H, T, D);
+    int st = ec::check_importance_args(Q, K, scores, lse, N, H, T, D, scale, ws, ws_bytes);
     if (st != EC_OK) return st;
-    if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
-    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(scores, 16) || (lse && !aligned(lse, 16))) return EC_ERR_ALIGN;
-    if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, T, D)) return EC_ERR_WORKSPACE;
-    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
     cudaError_t e = ec::launch_importance(Q, K, scores, lse, nullptr, N, H, T, 0, D, scale, EC_STAT_SUM, 0.0, ws,
                                           (cudaStream_t)stream);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
@@ -144,18 +201,9 @@ int ec_select_compact(const void *K, const void *V, const float *scores, int N, 
                       int share, int protect_ends, int compaction, void *Kc, void *Vc, int cap, int32_t *anchor_pos,
                       int32_t *bucket_len, void *ws, size_t ws_bytes, void *stream)
 {
-    if (!K || !V || !scores || !Kc || !Vc || !anchor_pos) return EC_ERR_NULL;
-    int st = check_shape(N, H, T, D);
+    int st = ec::check_select_compact_args(K, V, scores, N, H, T, D, n_keep, share, compaction, Kc, Vc, cap, anchor_pos,
+                                           bucket_len, ws, ws_bytes);
     if (st != EC_OK) return st;
-    if (n_keep < 1 || n_keep > T || cap < n_keep) return EC_ERR_ARG;
-    if (share < 1 || ((long long)N * H) % share != 0) return EC_ERR_ARG;
-    if (compaction != EC_COMPACT_MERGE && compaction != EC_COMPACT_EVICT) return EC_ERR_ARG;
-    if ((long long)N * H * cap >= (1LL << 31)) return EC_ERR_SHAPE;
-    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(scores, 4) ||
-        !aligned(anchor_pos, 4) || (bucket_len && !aligned(bucket_len, 4)))
-        return EC_ERR_ALIGN;
-    if (!ws || ws_bytes < ec_select_compact_workspace(N, H, T, D, n_keep, share)) return EC_ERR_WORKSPACE;
-    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
     float *mean_ws = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e = ec::launch_select(scores, N * H, T, n_keep, share, protect_ends ? 1 : 0, anchor_pos, bucket_len,
@@ -244,7 +292,9 @@ int ec_cache_init_ratio(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, in
 
 size_t ec_decode_workspace(const ec_cache *c)
 {
-    if (!c) return 0;
+    // shape fields only: the query is also made on a struct whose rows are not set up yet
+    if (!c || c->N < 1 || c->H < 1 || (c->D != 64 && c->D != 128) || c->cap < 1) return 0;
+    if ((long long)c->N * c->H >= (1LL << 24)) return 0;
     const int units = c->N * c->H;
     const int splits = ec::decode_splits(units, c->cap + 1);
     // arrival counters (one int per unit) followed by the per-split partial results
@@ -265,16 +315,9 @@ int decode_step_impl(const void *q, const void *k_new, const void *v_new, ec_cac
                      bool fresh_ws)
 {
     if (!q || !k_new || !v_new || !c || !out || !evicted_slot) return EC_ERR_NULL;
-    if (!c->Kc || !c->Vc) return EC_ERR_NULL;
+    int cst = ec::check_cache(c);
+    if (cst != EC_OK) return cst;
     const bool ratio = (c->policy == EC_POLICY_RATIO);
-    if (ratio) {
-        if (!c->recent_slots_host || c->offset < 1 || c->len < c->offset || c->len > c->cap || c->recent_head < 0 ||
-            c->recent_head >= c->offset || !(c->keep_ratio > 0.0 && c->keep_ratio <= 1.0))
-            return EC_ERR_ARG;
-    } else if (c->budget < 2 || c->budget > c->cap || c->len < 0 || c->len > c->budget || c->offset < 1 ||
-               c->offset > c->budget - 1 || c->ring_head < 0 || c->ring_head >= c->offset) {
-        return EC_ERR_ARG;
-    }
     if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
     if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16)) return EC_ERR_ALIGN;
     if (!ws || ws_bytes < ec_decode_workspace(c)) return EC_ERR_WORKSPACE;
@@ -347,7 +390,8 @@ int ec_decode_steps(const void *q, const void *k_new, const void *v_new, int ste
                     void *out, int *evicted_slots, void *ws, size_t ws_bytes, void *stream)
 {
     if (steps < 0) return EC_ERR_ARG;
-    if (!c) return EC_ERR_NULL;
+    int cst = ec::check_cache(c);
+    if (cst != EC_OK) return cst;
     const size_t stride = (size_t)c->N * c->H * c->D * 2;   // bytes of one [N, H, D] bf16 step
     // Rows no step of this call will write: new rows go to the slots of the `offset` most recent
     // rows (the ring of a full fixed-budget cache, the tracked recent slots of the ratio policy) or

@@ -55,6 +55,14 @@ __device__ __forceinline__ float fast_exp2(float x)
     return y;
 }
 
+// ---- host-only argument checks (ec_api.cu); each returns an ec_status ----
+int check_importance_args(const void *Q, const void *K, const float *scores, const float *lse, int N, int H, int T, int D,
+                          float scale, const void *ws, size_t ws_bytes);
+int check_select_compact_args(const void *K, const void *V, const float *scores, int N, int H, int T, int D, int n_keep,
+                              int share, int compaction, const void *Kc, const void *Vc, int cap,
+                              const int32_t *anchor_pos, const int32_t *bucket_len, const void *ws, size_t ws_bytes);
+int check_cache(const ec_cache *c);
+
 // ---- launchers implemented in the .cu files (all asynchronous on `stream`) ----
 cudaError_t launch_importance(const void *Q, const void *K, float *scores, float *lse_out, const float *lse_in,
                               int N, int H, int Tq, int P, int D, float scale, int statistic, double beta, void *ws,

@@ -321,6 +321,7 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
 int decode_splits(int units, int rows)
 {
     const int target = kMaxSplits;
+    if (units < 1) units = 1;
     int s = (target + units - 1) / units;
     int max_s = (rows + kMinRowsPerSplit - 1) / kMinRowsPerSplit;
     if (s > max_s) s = max_s;

@@ -45,7 +45,9 @@ size_t ec_decode_noalloc_capacity(void) { return kNoAllocBytes; }
 int ec_decode_step_noalloc(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale,
                            void *out, int *evicted_slot, int *slot_written, void *stream)
 {
-    if (!c) return EC_ERR_NULL;
+    // the caller owns *c: check it before anything is computed from its fields
+    int cst = ec::check_cache(c);
+    if (cst != EC_OK) return cst;
     // the same size rule as the ordinary call, measured against the fixed array
     const size_t need = ec_decode_workspace(c);
     if (need == 0 || need > kNoAllocBytes) return EC_ERR_TOO_LARGE;

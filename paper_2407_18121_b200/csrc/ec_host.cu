@@ -28,6 +28,13 @@ int ec_compress_host(const void *Q_host, const void *K_host, const void *V_host,
 {
     if (!Q_host || !K_host || !V_host || !Q_dev || !K_dev || !V_dev) return EC_ERR_NULL;
     if (N < 1 || H < 1 || T < 1 || (D != 64 && D != 128)) return EC_ERR_SHAPE;
+    if (population != EC_PER_HEAD && population != EC_LAYER_SHARED) return EC_ERR_ARG;
+    // everything the two device calls would reject is rejected here, before the first copy is enqueued
+    int pre = ec::check_importance_args(Q_dev, K_dev, scores_dev, nullptr, N, H, T, D, scale, ws_imp, ws_imp_bytes);
+    if (pre != EC_OK) return pre;
+    pre = ec::check_select_compact_args(K_dev, V_dev, scores_dev, N, H, T, D, n_keep, population == EC_LAYER_SHARED ? H : 1,
+                                        EC_COMPACT_MERGE, Kc_dev, Vc_dev, cap, anchor_pos_dev, nullptr, ws_sel, ws_sel_bytes);
+    if (pre != EC_OK) return pre;
     cudaStream_t s = (cudaStream_t)stream;
     const size_t bytes = (size_t)N * H * T * D * 2;
     if (cudaMemcpyAsync(Q_dev, Q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return EC_ERR_CUDA;
@@ -52,6 +59,16 @@ int ec_decode_steps_host(const void *q_host, const void *k_host, const void *v_h
     if (!q_host || !k_host || !v_host || !out_host || !q_dev || !k_dev || !v_dev || !out_dev || !c) return EC_ERR_NULL;
     if (!upload_stream || !download_stream) return EC_ERR_NULL;
     if (steps < 0 || chunk < 1) return EC_ERR_ARG;
+    // the cache struct, the scalar arguments and the workspace are checked before anything is enqueued;
+    // what can still fail later is a CUDA runtime call or, under the retention-ratio policy, a cache
+    // that has no room left to grow: c->step then tells how many steps were taken
+    int pre = ec::check_cache(c);
+    if (pre != EC_OK) return pre;
+    if (!(scale > 0.f) || !(scale < 3.0e38f)) return EC_ERR_ARG;
+    if (!ws || ws_bytes < ec_decode_workspace(c)) return EC_ERR_WORKSPACE;
+    if (((uintptr_t)ws & 255u) || ((uintptr_t)q_dev & 15u) || ((uintptr_t)k_dev & 15u) || ((uintptr_t)v_dev & 15u) ||
+        ((uintptr_t)out_dev & 15u))
+        return EC_ERR_ALIGN;
     if (steps == 0) return EC_OK;
     const int nchunks = (steps + chunk - 1) / chunk;
     if (2 * nchunks + 2 > 64) return EC_ERR_ARG;                       // at most 31 chunks per call

@@ -218,10 +218,13 @@ struct Geometry {
 };
 
 // How the attention rows are folded into a per-key statistic (Sec. 3.2 "Importance Metrics").
-// Query m enters pass 2 with weight 2^(wa + wb*m): pass 1 stores lse - (wa + wb*m), so the weight
-// costs nothing per element. wa = wb = 0 is the plain sum; a moving average with factor beta is
-// wa = log2(1-beta) + (Tq-1)*log2(beta), wb = -log2(beta). `mean` divides each key's total by the
-// number of queries that can see it.
+// Query m enters pass 2 with weight 2^(wa + wb*(m - (Tq-1))): pass 1 stores lse minus that exponent,
+// so the weight costs nothing per element. wa = wb = 0 is the plain sum; a moving average with
+// factor beta is wa = log2(1-beta), wb = -log2(beta). Counting from the last query keeps the exponent
+// small, hence exact to an fp32 ulp, for the newest queries, which are the ones whose weight matters
+// (for a long prompt and a small beta the oldest queries' exponents reach tens of thousands, but
+// their weights are zero to any precision). `mean` divides each key's total by the number of queries
+// that can see it.
 struct Fold {
     float wa, wb;
     int mean;
@@ -301,7 +304,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(bar_acc_full(b), 1);
             mbar_init(bar_acc_empty(b), 8);
-            mbar_init(bar_lse(b), 4 * 32);
+            mbar_init(bar_lse(b), 8 * 32);
         }
         mbar_init(bar_comb_full, 4 * 32);
         mbar_init(bar_comb_empty, 4 * 32);
@@ -429,13 +432,17 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (PASS2) {
                         // the first-half threads stage one entry each of the tile's lse (fetched one tile
                         // ahead, so its latency hides behind the previous tile's math), then all wait
-                        // (bounded) for the 128 entries; the buffer is reused two tiles later, after the
-                        // next tile's rendezvous
+                        // (bounded) for the 128 entries. Every softmax thread, readers of the second half
+                        // included, arrives on the tile's barrier: a thread that has passed the rendezvous
+                        // of tile t+1 therefore knows that all 256 have finished reading tile t's entries,
+                        // and only then may buffer b be overwritten for tile t+2.
                         if (half == 0) {
                             lse_s[b * kTileRows + r] = -lse_ahead;    // staged negated: exponent = v*c + (-lse)
                             mbar_arrive(bar_lse(b));
                             if (t + 1 < count)
                                 lse_ahead = lse2[lse_row + (size_t)stream_tile(first, t + 1) * kTileRows + r];
+                        } else {
+                            mbar_arrive(bar_lse(b));
                         }
                         if (!mbar_wait(bar_lse(b), bph, abort_flag, status)) { alive = false; break; }
                     }
@@ -530,7 +537,7 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         const float M = fmaxf(mrun, o.x);             // finite: column 0 of some tile is visible
                         const float Zs = Z * fast_exp2(mrun - M) + o.y * fast_exp2(o.x - M);
                         const float l2 = (row < geo.Tq) ? M + __log2f(Zs) : INFINITY;
-                        lse2[lse_row + row] = l2 - (fold.wa + fold.wb * (float)row);   // +inf stays +inf
+                        lse2[lse_row + row] = l2 - (fold.wa + fold.wb * (float)(row - (geo.Tq - 1)));   // +inf stays +inf
                         if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
                     } else if (row < Tk) {
                         float total = TAKE_MAX ? fmaxf(own, o.x) : own + o.x;
@@ -681,7 +688,7 @@ cudaError_t launch_importance(const void *Q, const void *K, float *scores, float
     Fold fold = {0.f, 0.f, statistic == EC_STAT_MEAN ? 1 : 0};
     if (statistic == EC_STAT_MOVING_AVERAGE) {
         const double lb = log2(beta);
-        fold.wa = (float)(log2(1.0 - beta) + (double)(Tq - 1) * lb);
+        fold.wa = (float)log2(1.0 - beta);
         fold.wb = (float)(-lb);
     }
     CUtensorMap mq, mk;

@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(G == 1 ? 128 : 32 * G)
 select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int protect_ends, int replicate,
               int32_t *__restrict__ anchor_pos, int32_t *__restrict__ bucket_len)
 {
-    __shared__ uint32_t xa[2][kMaxWarpsPerUnit], xc[2][kMaxWarpsPerUnit], xb[kMaxWarpsPerUnit];   // cross-warp exchange (G > 1)
+    __shared__ uint32_t xa[2][kMaxWarpsPerUnit], xc[2][kMaxWarpsPerUnit];   // cross-warp exchange (G > 1), double-buffered
     extern __shared__ uint32_t planes_all[];                               // 32 x 32 words per warp
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int unit = (G == 1) ? blockIdx.x * 4 + warp : blockIdx.x;
@@ -143,10 +143,10 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
     kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
     kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
     if (G > 1) {
-        if (lane == 0) { xa[par][wu] = kmin; xb[wu] = kmax; }
+        if (lane == 0) { xa[par][wu] = kmin; xc[par][wu] = kmax; }
         __syncthreads();
 #pragma unroll
-        for (int w = 0; w < G; ++w) { kmin = min(kmin, xa[par][w]); kmax = max(kmax, xb[w]); }
+        for (int w = 0; w < G; ++w) { kmin = min(kmin, xa[par][w]); kmax = max(kmax, xc[par][w]); }
         par ^= 1;
     }
     transpose32(pl);
@@ -196,11 +196,11 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
     if (G > 1) {
         const uint32_t gt = __reduce_add_sync(0xFFFFFFFFu, __popc(greater));
         const uint32_t eq = __reduce_add_sync(0xFFFFFFFFu, __popc(undecided));
-        if (lane == 0) { xa[par][wu] = gt; xb[wu] = eq; }
+        if (lane == 0) { xa[par][wu] = gt; xc[par][wu] = eq; }
         __syncthreads();
 #pragma unroll
         for (int w = 0; w < G; ++w)
-            if (w < wu) { gb += xa[par][w]; eb += xb[w]; }
+            if (w < wu) { gb += xa[par][w]; eb += xc[par][w]; }
         par ^= 1;
     }
 

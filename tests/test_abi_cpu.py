@@ -167,6 +167,63 @@ def test_select_compact_and_noalloc_validation(L):
     assert (big.len, big.step) == (128, 0)
 
 
+def test_a_zeroed_or_damaged_cache_struct_is_an_error_not_a_crash(L):
+    """The struct is caller-owned plain data: every call that reads one re-checks it."""
+    p = 0x10000
+    z = ec.ec_cache()                                   # all zero: N = H = 0 used to divide by zero
+    assert L.ec_decode_workspace(C.byref(z)) == 0
+    assert L.ec_decode_workspace(None) == 0
+    ev = C.c_int(0)
+    assert L.ec_decode_step_noalloc(p, p, p, C.byref(z), 1.0, p, C.byref(ev), None, None) == 1      # Kc, Vc NULL
+    assert L.ec_decode_step(p, p, p, C.byref(z), 1.0, p, C.byref(ev), None, p, 1 << 20, None) == 1
+    assert L.ec_decode_steps(p, p, p, 4, C.byref(z), 1.0, p, None, p, 1 << 20, None) == 1
+    c = ec.ec_cache()
+    assert L.ec_cache_init(C.byref(c), p, p, 2, 3, 64, 16, 8, 8, 4) == 0
+    for field, bad, want in (("N", 0, 2), ("H", -1, 2), ("D", 96, 2), ("cap", 0, 2), ("budget", 17, 4),
+                             ("ring_head", 4, 4), ("policy", 7, 4), ("offset", 0, 4), ("len", 9, 4)):
+        good = getattr(c, field)
+        setattr(c, field, bad)
+        assert L.ec_decode_step(p, p, p, C.byref(c), 1.0, p, C.byref(ev), None, p, 1 << 20, None) == want, field
+        assert L.ec_decode_step_noalloc(p, p, p, C.byref(c), 1.0, p, C.byref(ev), None, None) == want, field
+        setattr(c, field, good)
+    assert (c.len, c.step) == (8, 0)
+
+
+def test_host_tensor_calls_validate_before_enqueueing_anything(L):
+    """A rejected ec_compress_host / ec_decode_steps_host must not have started a copy: with no GPU in
+    this process any enqueued copy would surface as EC_ERR_CUDA (6) instead of the argument's code."""
+    p = 0x10000
+    ws = 1 << 22
+    f = L.ec_compress_host
+    ok_args = [p, p, p, p, p, p, p, 1, 2, 16, 64, 1.0, 8, 0, 1, p, p, 8, p, None, p, ws, p, ws, None]
+
+    def call(**change):
+        a = list(ok_args)
+        for k, v in change.items():
+            a[int(k[1:])] = v
+        return f(*a)
+
+    assert call(a11=0.0) == 4                       # scale
+    assert call(a12=17) == 4                        # n_keep > T
+    assert call(a17=4) == 4                         # cap < n_keep
+    assert call(a13=5) == 4                         # unknown population
+    assert call(a21=0) == 5                         # importance workspace too small
+    assert call(a23=0) == 5                         # selection workspace too small
+    assert call(a20=p + 16) == 3                    # workspace not 256-byte aligned
+    assert call(a3=p + 2) == 3                      # staging not 16-byte aligned
+    c = ec.ec_cache()
+    assert L.ec_cache_init(C.byref(c), p, p, 1, 2, 64, 16, 8, 8, 4) == 0
+    g = L.ec_decode_steps_host
+    one = 1
+    assert g(p, p, p, p, p, p, p, p, 4, 2, C.byref(c), 0.0, p, ws, None, one, one) == 4      # scale
+    assert g(p, p, p, p, p, p, p, p, 4, 2, C.byref(c), 1.0, p, 0, None, one, one) == 5       # workspace
+    assert g(p, p, p, p, p, p + 8, p, p, 4, 2, C.byref(c), 1.0, p, ws, None, one, one) == 3  # staging alignment
+    c.N = 0
+    assert g(p, p, p, p, p, p, p, p, 4, 2, C.byref(c), 1.0, p, ws, None, one, one) == 2      # damaged struct
+    c.N = 1
+    assert (c.len, c.step) == (8, 0)
+
+
 def test_header_is_plain_c(tmp_path):
     """ec.h is a C header: a C99 translation unit that includes nothing else compiles against it
     and can name every declared function with its declared type."""
