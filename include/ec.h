@@ -366,6 +366,25 @@ int ec_decode_steps_host(const void *q_host, const void *k_host, const void *v_h
 int ec_cache_concat(const ec_cache *c, const void *K_new_dev, const void *V_new_dev, int Tq,
                     void *K_all_dev, void *V_all_dev, void *stream);
 
+/* ---------------------------------------------------------------- measurement aids */
+
+/*
+ * (No counterpart in the paper.) Reads `bytes` of device memory once with 16-byte streaming loads
+ * and folds them into *sink_dev with XOR, so that timing the call gives the read-only bandwidth
+ * this GPU sustains: the ceiling for the decode and merge kernels, which read far more than
+ * they write (a copy, half reads and half writes, runs below it).
+ *   buf_dev    device, 16-byte aligned, `bytes` long (bytes >= 16, a multiple of 16)
+ *   sink_dev   device uint32, read-modify-written
+ */
+int ec_probe_read_stream(const void *buf_dev, size_t bytes, unsigned *sink_dev, void *stream);
+
+/*
+ * How many CTAs would share one unit's rows if ec_decode_step were called on *c now (1: one
+ * CTA per unit, the layout of large batches; > 1: the split path with in-kernel merge).
+ * 0 when *c is invalid.
+ */
+int ec_decode_splits(const ec_cache *c);
+
 /* ---------------------------------------------------------------- no-allocation decode */
 
 /*

@@ -28,6 +28,7 @@ EXPORTS = (
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
     "ec_cache_init", "ec_cache_init_ratio", "ec_cache_concat", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc", "ec_compress_host", "ec_decode_steps_host",
+    "ec_probe_read_stream", "ec_decode_splits",
 )
 
 
@@ -107,6 +108,10 @@ def lib() -> C.CDLL:
     L.ec_decode_noalloc_capacity.argtypes = []
     L.ec_decode_step_noalloc.restype = i
     L.ec_decode_step_noalloc.argtypes = [vp, vp, vp, C.POINTER(ec_cache), f, vp, C.POINTER(i), C.POINTER(i), vp]
+    L.ec_probe_read_stream.restype = i
+    L.ec_probe_read_stream.argtypes = [vp, sz, vp, vp]
+    L.ec_decode_splits.restype = i
+    L.ec_decode_splits.argtypes = [C.POINTER(ec_cache)]
     _lib = L
     return L
 
@@ -337,3 +342,13 @@ def ec_decode_steps_host(q_host, k_host, v_host, out_host, q, k, v, out, cache: 
                                     float(scale), _ptr(ws), ws.numel() * ws.element_size(), _stream(),
                                     upload_stream.cuda_stream, download_stream.cuda_stream)
     _check(st, "ec_decode_steps_host")
+
+
+def ec_probe_read_stream(buf: torch.Tensor, sink: torch.Tensor) -> None:
+    """Enqueue one read-only pass over `buf` (any dtype, byte size a multiple of 16); `sink`: uint32/int32 [1]."""
+    _check(lib().ec_probe_read_stream(_ptr(buf), buf.numel() * buf.element_size(), _ptr(sink), _stream()),
+           "ec_probe_read_stream")
+
+
+def ec_decode_splits(cache: ec_cache) -> int:
+    return int(lib().ec_decode_splits(C.byref(cache)))
