@@ -342,17 +342,14 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            uint32_t armed = 0;
+            uint32_t armed = 0, stat_armed = 0;           // streamed tiles / stationary tiles whose copies were started
             for (int round = 0, sidx; alive && (sidx = pair_of_round(round)) >= 0; ++round) {
                 for (int sub = 0; alive && sub < 2; ++sub) {
                     int unit, st, first, count;
                     if (!item_of(sidx, sub, unit, st, first, count)) break;
-                    // the stationary buffer is free once the previous item's last MMA has completed
-                    if (!mbar_wait(bar_stat_empty, (it + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                    mbar_expect_tx(bar_stat_full, kTileBytes);
-#pragma unroll
-                    for (int bx = 0; bx < kBoxes; ++bx)
-                        tma_load_3d(base + L::kStat + bx * kBoxBytes, map_stat, bx * 64, st * kTileRows, unit, bar_stat_full);
+                    // The item's first streamed tile goes out first: its ring stage was released by an
+                    // earlier MMA of the previous item, whereas the stationary buffer is free only once
+                    // that item's last MMA has completed.
                     for (int t = 0; t < count; ++t, ++tg) {
                         const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
                         if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
@@ -362,13 +359,21 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             tma_load_3d(base + L::kStage0 + s * kTileBytes + bx * kBoxBytes, map_strm, bx * 64,
                                         stream_tile(first, t) * kTileRows, unit, bar_full(s));
                         armed = tg + 1;
+                        if (t == 0) {
+                            if (!mbar_wait(bar_stat_empty, (it + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                            mbar_expect_tx(bar_stat_full, kTileBytes);
+#pragma unroll
+                            for (int bx = 0; bx < kBoxes; ++bx)
+                                tma_load_3d(base + L::kStat + bx * kBoxBytes, map_stat, bx * 64, st * kTileRows, unit, bar_stat_full);
+                            stat_armed = it + 1;
+                        }
                     }
                     ++it;
                 }
             }
             if (*abort_flag) {
                 // let copies that are still in flight land before the CTA gives its memory back
-                if (it > 0) mbar_wait(bar_stat_full, (it - 1u) & 1u, abort_flag, status, 200000ull);
+                if (stat_armed > 0) mbar_wait(bar_stat_full, (stat_armed - 1u) & 1u, abort_flag, status, 200000ull);
                 for (uint32_t t = armed > (uint32_t)STAGES ? armed - STAGES : 0; t < armed; ++t)
                     mbar_wait(bar_full(t % STAGES), (t / STAGES) & 1u, abort_flag, status, 200000ull);
             }
@@ -500,20 +505,44 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         }
                     };
 
-                    // this thread's 64 columns: the second 32 are in flight while the first are processed.
                     // Only tiles the diagonal crosses pay for the mask: they run a separate instance.
                     auto tile_body = [&](auto mask_tag) {
+                        constexpr bool MASKED = decltype(mask_tag)::value;
                         const uint32_t col0 = lane_addr + b * kTileRows;
-                        uint32_t ra[32], rb[32];
-                        tmem_ld32_async(col0, ra);
-                        tmem_ld_wait(ra);
-                        tmem_ld32_async(col0 + 32, rb);
-                        chunk(ra, half * 2, mask_tag);
-                        tmem_ld_wait(rb);
-                        tc_fence_before();                   // all TMEM reads of this tile are done:
-                        __syncwarp();                        // hand the accumulator back before the last chunk's math
-                        if (lane == 0) mbar_arrive(bar_acc_empty(b));
-                        chunk(rb, half * 2 + 1, mask_tag);
+                        // A chunk the mask hides from all 32 rows of this warp is neither read nor
+                        // exponentiated (on a diagonal tile that is 6 of the 16 warp x chunk blocks).
+                        //   pass 1: column visible iff col <= row + off  -> hidden iff first col > last row + off
+                        //   pass 2: column visible iff col >= row - off  -> hidden iff last col < first row - off
+                        auto hidden = [&](int ch) {
+                            if (!MASKED) return false;
+                            return PASS2 ? (ch * 32 + 31 < q4 * 32 - off) : (ch * 32 > q4 * 32 + 31 + off);
+                        };
+                        const bool skip_a = hidden(half * 2), skip_b = hidden(half * 2 + 1);   // warp-uniform
+                        auto release = [&]() {
+                            tc_fence_before();               // all TMEM reads of this tile are done:
+                            __syncwarp();                    // hand the accumulator back before the last chunk's math
+                            if (lane == 0) mbar_arrive(bar_acc_empty(b));
+                        };
+                        if (!skip_a && !skip_b) {
+                            // this thread's 64 columns: the second 32 are in flight while the first are processed
+                            uint32_t ra[32], rb[32];
+                            tmem_ld32_async(col0, ra);
+                            tmem_ld_wait(ra);
+                            tmem_ld32_async(col0 + 32, rb);
+                            chunk(ra, half * 2, mask_tag);
+                            tmem_ld_wait(rb);
+                            release();
+                            chunk(rb, half * 2 + 1, mask_tag);
+                        } else if (skip_a && skip_b) {
+                            release();
+                        } else {
+                            const int which = skip_a ? 1 : 0;     // the one chunk some row of the warp can see
+                            uint32_t ra[32];
+                            tmem_ld32_async(col0 + 32 * which, ra);
+                            tmem_ld_wait(ra);
+                            release();
+                            chunk(ra, half * 2 + which, mask_tag);
+                        }
                     };
                     if (masked) tile_body(std::true_type{});
                     else tile_body(std::false_type{});
