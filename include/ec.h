@@ -241,6 +241,8 @@ typedef struct {
     int64_t n_tot;      /* tokens seen so far, prompt included                           */
     int *recent_slots_host; /* caller-owned host array of `offset` ints: physical slots
                                of the `offset` newest rows, kept as a ring               */
+    int *queue_slots_host;  /* optional (see ec_cache_track_order): caller-owned host array
+                               of `cap` ints, the physical slot of every row in queue order */
 } ec_cache;
 
 typedef enum {
@@ -270,6 +272,21 @@ int ec_cache_init_ratio(ec_cache *c, void *Kc_dev, void *Vc_dev, int N, int H, i
 /* Bytes of device scratch the decode calls need for this cache; depends on N, H, D and cap only.
  * 0 when those fields are out of range (N, H, cap >= 1; D 64 or 128; N*H < 2^24) or c is NULL. */
 size_t ec_decode_workspace(const ec_cache *c);
+
+/*
+ * Makes a retention-ratio cache remember its queue order, so that a further instruction can be
+ * encoded on top of it (ec_cache_concat). Under that policy a new row is appended while the cache
+ * may grow and otherwise takes the slot of the row that leaves, so physical order and queue order
+ * drift apart in a way only the sequence of grow / evict decisions determines; every decode step
+ * then updates the list (an O(offset) shift on the host).
+ *   c                  EC_POLICY_RATIO cache on which no step has been taken yet (c->step == 0):
+ *                      its rows are still in slot order
+ *   queue_slots_host   host array of c->cap ints owned by the caller, valid as long as *c is used;
+ *                      entries 0 .. len-1 are filled here with 0 .. len-1
+ * Returns EC_ERR_ARG for a fixed-budget cache (its order is implied by budget, offset and
+ * ring_head) or when steps were already taken.
+ */
+int ec_cache_track_order(ec_cache *c, int *queue_slots_host);
 
 /*
  * One generation step (Sec. 3.3 "Output Generation"; Algorithm 1, last branch):
@@ -353,15 +370,17 @@ int ec_decode_steps_host(const void *q_host, const void *k_host, const void *v_h
  * stage takes in the chat history): the cache's rows in queue order, oldest first, followed
  * by the Tq rows of the new tokens. The result feeds ec_importance_prefix (P = c->len) and
  * ec_select_merge / ec_select_compact over T = c->len + Tq rows.
- *   c                      fixed-budget cache (EC_POLICY_FIXED; the retention-ratio policy does
- *                          not keep the queue order of old rows and returns EC_ERR_ARG);
- *                          read only, c->len >= 1
+ *   c                      fixed-budget cache, or a retention-ratio cache that tracks its queue
+ *                          order (ec_cache_track_order; without it EC_ERR_ARG); read only,
+ *                          c->len >= 1
  *   K_new_dev, V_new_dev   device bf16 [N, H, Tq, D], 16-byte aligned, Tq >= 1
  *   K_all_dev, V_all_dev   device bf16 [N, H, c->len + Tq, D], written; must not overlap
  *                          the cache or the new rows
  * Row j < len of a unit comes from physical slot j while j < budget - offset or the cache is
  * not yet full, else from the ring: slot (budget - offset) + (ring_head + j - (budget - offset))
- * mod offset. Rows are copied bit for bit. Asynchronous on `stream`.
+ * mod offset; for a retention-ratio cache from slot queue_slots_host[j] (the list is passed to
+ * the copy kernels by value, a few hundred rows per launch, so the host array may change as soon
+ * as the call returns). Rows are copied bit for bit. Asynchronous on `stream`.
  */
 int ec_cache_concat(const ec_cache *c, const void *K_new_dev, const void *V_new_dev, int Tq,
                     void *K_all_dev, void *V_all_dev, void *stream);

@@ -26,7 +26,7 @@ EXPORTS = (
     "ec_status_string", "ec_keep_count",
     "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_statistic", "ec_importance_from_lse", "ec_device_status", "ec_selftest_wait_timeout",
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
-    "ec_cache_init", "ec_cache_init_ratio", "ec_cache_concat", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
+    "ec_cache_init", "ec_cache_init_ratio", "ec_cache_track_order", "ec_cache_concat", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc", "ec_compress_host", "ec_decode_steps_host",
     "ec_probe_read_stream", "ec_decode_splits",
 )
@@ -45,7 +45,8 @@ class ec_cache(C.Structure):
                 ("len", C.c_int), ("budget", C.c_int), ("offset", C.c_int),
                 ("ring_head", C.c_int), ("step", C.c_int64),
                 ("policy", C.c_int), ("recent_head", C.c_int), ("keep_ratio", C.c_double),
-                ("n_tot", C.c_int64), ("recent_slots_host", C.POINTER(C.c_int))]
+                ("n_tot", C.c_int64), ("recent_slots_host", C.POINTER(C.c_int)),
+                ("queue_slots_host", C.POINTER(C.c_int))]
 
 
 _lib = None
@@ -92,6 +93,8 @@ def lib() -> C.CDLL:
     L.ec_cache_init_ratio.restype = i
     L.ec_cache_init_ratio.argtypes = [C.POINTER(ec_cache), vp, vp, i, i, i, i, i, i, C.c_double, C.c_int64,
                                       C.POINTER(C.c_int)]
+    L.ec_cache_track_order.restype = i
+    L.ec_cache_track_order.argtypes = [C.POINTER(ec_cache), C.POINTER(C.c_int)]
     L.ec_cache_concat.restype = i
     L.ec_cache_concat.argtypes = [C.POINTER(ec_cache), vp, vp, i, vp, vp, vp]
     L.ec_decode_workspace.restype = sz
@@ -245,16 +248,20 @@ def ec_cache_init(Kc: torch.Tensor, Vc: torch.Tensor, length: int, budget: int, 
 
 
 def ec_cache_init_ratio(Kc: torch.Tensor, Vc: torch.Tensor, length: int, offset: int, keep_ratio: float,
-                        n_tot: int) -> ec_cache:
+                        n_tot: int, track_order: bool = True) -> ec_cache:
     """Cache under the retention-ratio policy: it grows while length < keep_ratio * tokens seen and
     evicts at the fixed truncation location otherwise. The host ring of recent slots is owned by
-    the returned object."""
+    the returned object, and so is the queue-order list that ec_cache_track_order maintains (needed
+    by ec_cache_concat; `track_order=False` leaves it out)."""
     N, H, cap, D = Kc.shape
     c = ec_cache()
     c._recent = (C.c_int * int(offset))()          # kept alive with the struct
     st = lib().ec_cache_init_ratio(C.byref(c), _ptr(Kc), _ptr(Vc), N, H, D, cap, int(length), int(offset),
                                    float(keep_ratio), int(n_tot), c._recent)
     _check(st, "ec_cache_init_ratio")
+    if track_order:
+        c._order = (C.c_int * int(cap))()          # queue order of the rows, kept alive with the struct
+        _check(lib().ec_cache_track_order(C.byref(c), c._order), "ec_cache_track_order")
     return c
 
 

@@ -124,6 +124,7 @@ size_t ec_importance_workspace(int N, int H, int T, int D)
 int ec_importance(const void *Q, const void *K, float *scores, float *lse, int N, int H, int T, int D,
                   float scale, void *ws, size_t ws_bytes, void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_importance");
     int st = ec::check_importance_args(Q, K, scores, lse, N, H, T, D, scale, ws, ws_bytes);
     if (st != EC_OK) return st;
     cudaError_t e = ec::launch_importance(Q, K, scores, lse, nullptr, N, H, T, 0, D, scale, EC_STAT_SUM, 0.0, ws,
@@ -134,6 +135,7 @@ int ec_importance(const void *Q, const void *K, float *scores, float *lse, int N
 int ec_importance_statistic(const void *Q, const void *K, float *scores, float *lse, int N, int H, int Tq, int P, int D,
                             float scale, int statistic, double beta, void *ws, size_t ws_bytes, void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_importance_statistic");
     if (!Q || !K || !scores) return EC_ERR_NULL;
     if (P < 0 || Tq < 1 || (long long)P + Tq > kMaxT) return EC_ERR_SHAPE;
     int st = check_shape(N, H, Tq + P, D);
@@ -158,6 +160,7 @@ int ec_importance_prefix(const void *Q, const void *K, float *scores, float *lse
 int ec_importance_from_lse(const void *Q, const void *K, const float *lse, float *scores, int N, int H, int T, int D,
                            float scale, void *ws, size_t ws_bytes, void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_importance_from_lse");
     if (!Q || !K || !scores || !lse) return EC_ERR_NULL;
     int st = check_shape(N, H, T, D);
     if (st != EC_OK) return st;
@@ -201,6 +204,7 @@ int ec_select_compact(const void *K, const void *V, const float *scores, int N, 
                       int share, int protect_ends, int compaction, void *Kc, void *Vc, int cap, int32_t *anchor_pos,
                       int32_t *bucket_len, void *ws, size_t ws_bytes, void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_select_compact");
     int st = ec::check_select_compact_args(K, V, scores, N, H, T, D, n_keep, share, compaction, Kc, Vc, cap, anchor_pos,
                                            bucket_len, ws, ws_bytes);
     if (st != EC_OK) return st;
@@ -246,24 +250,34 @@ int ec_cache_init(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, int cap,
     c->keep_ratio = 0.0;
     c->n_tot = 0;
     c->recent_slots_host = nullptr;
+    c->queue_slots_host = nullptr;
     return EC_OK;
 }
 
 int ec_cache_concat(const ec_cache *c, const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
                     void *stream)
 {
-    if (!c || !K_new || !V_new || !K_all || !V_all || !c->Kc || !c->Vc) return EC_ERR_NULL;
-    if (c->policy != EC_POLICY_FIXED) return EC_ERR_ARG;
-    if (c->N < 1 || c->H < 1 || (c->D != 64 && c->D != 128)) return EC_ERR_SHAPE;
-    if (Tq < 1 || c->len < 1 || c->len > c->budget || c->budget > c->cap) return EC_ERR_ARG;
-    if (c->offset < 1 || c->offset > c->budget - 1 || c->ring_head < 0 || c->ring_head >= c->offset) return EC_ERR_ARG;
+    ec::NvtxRange nvtx_range("ec_cache_concat");
+    if (!c || !K_new || !V_new || !K_all || !V_all) return EC_ERR_NULL;
+    int st = ec::check_cache(c);
+    if (st != EC_OK) return st;
+    if (c->policy == EC_POLICY_RATIO && !c->queue_slots_host) return EC_ERR_ARG;   // order not tracked
+    if (Tq < 1 || c->len < 1) return EC_ERR_ARG;
     const long long units = (long long)c->N * c->H;
     if (units * ((long long)c->len + Tq) >= (1LL << 31)) return EC_ERR_SHAPE;
     if (!aligned(K_new, 16) || !aligned(V_new, 16) || !aligned(K_all, 16) || !aligned(V_all, 16)) return EC_ERR_ALIGN;
-    const bool full = c->len == c->budget;               // the ring exists once the cache has reached its budget
-    cudaError_t e = ec::launch_concat(c->Kc, c->Vc, (int)units, c->cap, c->D, c->len, full ? c->budget - c->offset : c->len,
-                                      full ? c->offset : 0, full ? c->ring_head : 0, K_new, V_new, Tq, K_all, V_all,
-                                      (cudaStream_t)stream);
+    cudaError_t e;
+    if (c->policy == EC_POLICY_RATIO) {
+        for (int j = 0; j < c->len; ++j)
+            if (c->queue_slots_host[j] < 0 || c->queue_slots_host[j] >= c->cap) return EC_ERR_ARG;
+        e = ec::launch_concat_listed(c->Kc, c->Vc, (int)units, c->cap, c->D, c->len, c->queue_slots_host, K_new, V_new, Tq,
+                                     K_all, V_all, (cudaStream_t)stream);
+    } else {
+        const bool full = c->len == c->budget;           // the ring exists once the cache has reached its budget
+        e = ec::launch_concat(c->Kc, c->Vc, (int)units, c->cap, c->D, c->len, full ? c->budget - c->offset : c->len,
+                              full ? c->offset : 0, full ? c->ring_head : 0, K_new, V_new, Tq, K_all, V_all,
+                              (cudaStream_t)stream);
+    }
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 
@@ -286,7 +300,19 @@ int ec_cache_init_ratio(ec_cache *c, void *Kc, void *Vc, int N, int H, int D, in
     c->keep_ratio = keep_ratio;
     c->n_tot = n_tot;
     c->recent_slots_host = recent_slots;
+    c->queue_slots_host = nullptr;
     for (int i = 0; i < offset; ++i) recent_slots[i] = len - offset + i;   // oldest first
+    return EC_OK;
+}
+
+int ec_cache_track_order(ec_cache *c, int *queue_slots)
+{
+    if (!c || !queue_slots) return EC_ERR_NULL;
+    int st = ec::check_cache(c);
+    if (st != EC_OK) return st;
+    if (c->policy != EC_POLICY_RATIO || c->step != 0) return EC_ERR_ARG;
+    for (int i = 0; i < c->len; ++i) queue_slots[i] = i;
+    c->queue_slots_host = queue_slots;
     return EC_OK;
 }
 
@@ -360,6 +386,17 @@ int decode_step_impl(const void *q, const void *k_new, const void *v_new, ec_cac
                           partials, counters, splits, (cudaStream_t)stream);
     if (e != cudaSuccess) return EC_ERR_CUDA;
     if (ratio) {
+        if (c->queue_slots_host) {
+            // queue order: the row that leaves sits `offset` places before the end (it is the oldest of
+            // the `offset` newest rows); the rows behind it move up, the new row joins at the tail
+            int *order = c->queue_slots_host;
+            if (evicted >= 0) {
+                for (int j = c->len - c->offset; j < c->len - 1; ++j) order[j] = order[j + 1];
+                order[c->len - 1] = slot;
+            } else {
+                order[c->len] = slot;
+            }
+        }
         // the new row is now the newest; the ring's oldest entry either left or stops being tracked
         c->recent_slots_host[c->recent_head] = slot;
         c->recent_head = (c->recent_head + 1) % c->offset;
@@ -383,12 +420,14 @@ extern "C" {
 int ec_decode_step(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale, void *out,
                    int *evicted_slot, int *slot_written, void *ws, size_t ws_bytes, void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_decode_step");
     return decode_step_impl(q, k_new, v_new, c, scale, out, evicted_slot, slot_written, ws, ws_bytes, stream, -1, true);
 }
 
 int ec_decode_steps(const void *q, const void *k_new, const void *v_new, int steps, ec_cache *c, float scale,
                     void *out, int *evicted_slots, void *ws, size_t ws_bytes, void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_decode_steps");
     if (steps < 0) return EC_ERR_ARG;
     int cst = ec::check_cache(c);
     if (cst != EC_OK) return cst;

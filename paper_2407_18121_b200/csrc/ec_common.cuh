@@ -5,9 +5,20 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "ec.h"
 
 namespace ec {
+
+// A named range around every entry point that enqueues work, visible to profilers that listen to
+// NVTX (header-only: without such a tool attached the calls return at once).
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
 
 constexpr int kStatusBytes = 256;   // status block at the head of an importance workspace
 
@@ -80,6 +91,10 @@ cudaError_t launch_gather(const void *K, const void *V, const int32_t *anchor_po
 cudaError_t launch_concat(const void *Kc, const void *Vc, int units, int cap, int D, int P, int base, int ring,
                           int ring_head, const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
                           cudaStream_t stream);
+// The same with the cache rows' slots given as a host list: queue position j comes from slot slots[j].
+cudaError_t launch_concat_listed(const void *Kc, const void *Vc, int units, int cap, int D, int P, const int *slots_host,
+                                 const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
+                                 cudaStream_t stream);
 cudaError_t launch_merge(const void *K, const void *V, const int32_t *anchor_pos, int units, int T, int D,
                          int n_keep, void *Kc, void *Vc, int cap, cudaStream_t stream);
 

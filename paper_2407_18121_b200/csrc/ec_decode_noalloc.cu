@@ -45,6 +45,7 @@ size_t ec_decode_noalloc_capacity(void) { return kNoAllocBytes; }
 int ec_decode_step_noalloc(const void *q, const void *k_new, const void *v_new, ec_cache *c, float scale,
                            void *out, int *evicted_slot, int *slot_written, void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_decode_step_noalloc");
     // the caller owns *c: check it before anything is computed from its fields
     int cst = ec::check_cache(c);
     if (cst != EC_OK) return cst;

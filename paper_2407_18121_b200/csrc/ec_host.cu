@@ -26,6 +26,7 @@ int ec_compress_host(const void *Q_host, const void *K_host, const void *V_host,
                      int32_t *anchor_pos_host, void *ws_imp, size_t ws_imp_bytes, void *ws_sel, size_t ws_sel_bytes,
                      void *stream)
 {
+    ec::NvtxRange nvtx_range("ec_compress_host");
     if (!Q_host || !K_host || !V_host || !Q_dev || !K_dev || !V_dev) return EC_ERR_NULL;
     if (N < 1 || H < 1 || T < 1 || (D != 64 && D != 128)) return EC_ERR_SHAPE;
     if (population != EC_PER_HEAD && population != EC_LAYER_SHARED) return EC_ERR_ARG;
@@ -56,6 +57,7 @@ int ec_decode_steps_host(const void *q_host, const void *k_host, const void *v_h
                          void *k_dev, void *v_dev, void *out_dev, int steps, int chunk, ec_cache *c, float scale,
                          void *ws, size_t ws_bytes, void *stream, void *upload_stream, void *download_stream)
 {
+    ec::NvtxRange nvtx_range("ec_decode_steps_host");
     if (!q_host || !k_host || !v_host || !out_host || !q_dev || !k_dev || !v_dev || !out_dev || !c) return EC_ERR_NULL;
     if (!upload_stream || !download_stream) return EC_ERR_NULL;
     if (steps < 0 || chunk < 1) return EC_ERR_ARG;

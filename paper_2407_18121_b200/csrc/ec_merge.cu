@@ -149,10 +149,11 @@ gather_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const in
 
 // History for a further instruction: output row j of a unit is cache row j in queue order for
 // j < P, new row j - P after it. One lane group per output row, K on its first half, V on the second.
+// The launch covers output rows row0 .. P + Tq - 1.
 template <int LPR>
 __global__ void __launch_bounds__(kMergeThreads)
 concat_kernel(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, int cap, int P, int base, int ring,
-              int ring_head, const uint4 *__restrict__ K_new, const uint4 *__restrict__ V_new, int Tq, int chunks,
+              int ring_head, const uint4 *__restrict__ K_new, const uint4 *__restrict__ V_new, int Tq, int row0, int chunks,
               uint4 *__restrict__ K_all, uint4 *__restrict__ V_all)
 {
     constexpr int GL = 2 * LPR;
@@ -162,7 +163,7 @@ concat_kernel(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, int ca
     const int g = threadIdx.x / GL, gl = threadIdx.x - g * GL;
     const bool is_v = gl >= LPR;
     const int l = is_v ? gl - LPR : gl;
-    const int j = chunk * G + g;
+    const int j = row0 + chunk * G + g;
     const int T = P + Tq;
     if (j >= T) return;
     const uint4 *src;
@@ -173,6 +174,30 @@ concat_kernel(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, int ca
         src = (is_v ? V_new : K_new) + ((size_t)unit * Tq + (j - P)) * LPR + l;
     }
     uint4 *dst = (is_v ? V_all : K_all) + ((size_t)unit * T + j) * LPR + l;
+    *dst = ldg_stream(src);
+}
+
+// Cache rows whose slots follow no formula (retention-ratio policy): output rows j0 .. j0 + n - 1 of
+// every unit come from the slots listed in `tab`, which travels by value in the kernel's parameters.
+constexpr int kSlotTableRows = 896;
+struct SlotTable { int slot[kSlotTableRows]; };
+
+template <int LPR>
+__global__ void __launch_bounds__(kMergeThreads)
+concat_listed_kernel(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, int cap, int T_out, int j0, int n,
+                     const __grid_constant__ SlotTable tab, int chunks, uint4 *__restrict__ K_all, uint4 *__restrict__ V_all)
+{
+    constexpr int GL = 2 * LPR;
+    constexpr int G = kMergeThreads / GL;
+    const int unit = blockIdx.x / chunks;
+    const int chunk = blockIdx.x - unit * chunks;
+    const int g = threadIdx.x / GL, gl = threadIdx.x - g * GL;
+    const bool is_v = gl >= LPR;
+    const int l = is_v ? gl - LPR : gl;
+    const int j = chunk * G + g;
+    if (j >= n) return;
+    const uint4 *src = (is_v ? Vc : Kc) + ((size_t)unit * cap + tab.slot[j]) * LPR + l;
+    uint4 *dst = (is_v ? V_all : K_all) + ((size_t)unit * T_out + j0 + j) * LPR + l;
     *dst = ldg_stream(src);
 }
 
@@ -222,15 +247,40 @@ cudaError_t launch_gather_t(const void *K, const void *V, const int32_t *anchor_
 
 template <int LPR>
 cudaError_t launch_concat_t(const void *Kc, const void *Vc, int units, int cap, int P, int base, int ring, int ring_head,
-                            const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all, cudaStream_t stream)
+                            const void *K_new, const void *V_new, int Tq, int row0, void *K_all, void *V_all,
+                            cudaStream_t stream)
 {
     constexpr int G = kMergeThreads / (2 * LPR);
-    const int chunks = (P + Tq + G - 1) / G;
+    const int chunks = (P + Tq - row0 + G - 1) / G;
     if ((long long)units * chunks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     concat_kernel<LPR><<<(unsigned)(units * chunks), kMergeThreads, 0, stream>>>(
         (const uint4 *)Kc, (const uint4 *)Vc, cap, P, base, ring, ring_head, (const uint4 *)K_new, (const uint4 *)V_new, Tq,
-        chunks, (uint4 *)K_all, (uint4 *)V_all);
+        row0, chunks, (uint4 *)K_all, (uint4 *)V_all);
     return cudaGetLastError();
+}
+
+template <int LPR>
+cudaError_t launch_concat_listed_t(const void *Kc, const void *Vc, int units, int cap, int P, const int *slots,
+                                   const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
+                                   cudaStream_t stream)
+{
+    constexpr int G = kMergeThreads / (2 * LPR);
+    // the new rows: the plain kernel from output row P on
+    cudaError_t e = launch_concat_t<LPR>(Kc, Vc, units, cap, P, P, 0, 0, K_new, V_new, Tq, P, K_all, V_all, stream);
+    if (e != cudaSuccess) return e;
+    for (int j0 = 0; j0 < P; j0 += kSlotTableRows) {
+        const int n = P - j0 < kSlotTableRows ? P - j0 : kSlotTableRows;
+        SlotTable tab;
+        for (int j = 0; j < n; ++j) tab.slot[j] = slots[j0 + j];
+        for (int j = n; j < kSlotTableRows; ++j) tab.slot[j] = 0;
+        const int chunks = (n + G - 1) / G;
+        if ((long long)units * chunks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+        concat_listed_kernel<LPR><<<(unsigned)(units * chunks), kMergeThreads, 0, stream>>>(
+            (const uint4 *)Kc, (const uint4 *)Vc, cap, P + Tq, j0, n, tab, chunks, (uint4 *)K_all, (uint4 *)V_all);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -257,8 +307,17 @@ cudaError_t launch_concat(const void *Kc, const void *Vc, int units, int cap, in
                           cudaStream_t stream)
 {
     if (D == 128)
-        return launch_concat_t<16>(Kc, Vc, units, cap, P, base, ring, ring_head, K_new, V_new, Tq, K_all, V_all, stream);
-    return launch_concat_t<8>(Kc, Vc, units, cap, P, base, ring, ring_head, K_new, V_new, Tq, K_all, V_all, stream);
+        return launch_concat_t<16>(Kc, Vc, units, cap, P, base, ring, ring_head, K_new, V_new, Tq, 0, K_all, V_all, stream);
+    return launch_concat_t<8>(Kc, Vc, units, cap, P, base, ring, ring_head, K_new, V_new, Tq, 0, K_all, V_all, stream);
+}
+
+cudaError_t launch_concat_listed(const void *Kc, const void *Vc, int units, int cap, int D, int P, const int *slots_host,
+                                 const void *K_new, const void *V_new, int Tq, void *K_all, void *V_all,
+                                 cudaStream_t stream)
+{
+    if (D == 128)
+        return launch_concat_listed_t<16>(Kc, Vc, units, cap, P, slots_host, K_new, V_new, Tq, K_all, V_all, stream);
+    return launch_concat_listed_t<8>(Kc, Vc, units, cap, P, slots_host, K_new, V_new, Tq, K_all, V_all, stream);
 }
 
 }  // namespace ec

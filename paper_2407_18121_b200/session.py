@@ -63,12 +63,14 @@ class ElasticCacheSession:
 
     # ---- a new instruction on top of the current cache ---------------------------------
     def logical_slots(self):
-        """Physical slots of the cache rows in queue order (oldest first), fixed-budget policy:
-        the rows before the ring never move; the ring holds the `offset` newest rows, oldest at
-        `ring_head`."""
+        """Physical slots of the cache rows in queue order (oldest first). Fixed budget: the rows
+        before the ring never move; the ring holds the `offset` newest rows, oldest at `ring_head`.
+        Retention ratio: the list the library maintains (ec_cache_track_order)."""
         c = self.cache
         if c.policy != 0:
-            raise ValueError("queue order is only tracked for the fixed-budget policy")
+            if not c.queue_slots_host:
+                raise ValueError("this retention-ratio cache does not track its queue order")
+            return [c.queue_slots_host[j] for j in range(c.len)]
         if c.len < c.budget:
             return list(range(c.len))
         base = c.budget - c.offset

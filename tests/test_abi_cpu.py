@@ -167,6 +167,23 @@ def test_select_compact_and_noalloc_validation(L):
     assert (big.len, big.step) == (128, 0)
 
 
+def test_queue_order_tracking_validation(L):
+    p = 0x10000
+    c = ec.ec_cache()
+    ring = (C.c_int * 8)()
+    order = (C.c_int * 64)()
+    assert L.ec_cache_init_ratio(C.byref(c), p, p, 1, 2, 64, 64, 20, 8, 0.5, 40, ring) == 0
+    assert not c.queue_slots_host
+    assert L.ec_cache_track_order(C.byref(c), None) == 1
+    assert L.ec_cache_track_order(C.byref(c), order) == 0
+    assert list(order)[:20] == list(range(20))
+    c.step = 3
+    assert L.ec_cache_track_order(C.byref(c), order) == 4            # rows may no longer be in slot order
+    fixed = ec.ec_cache()
+    assert L.ec_cache_init(C.byref(fixed), p, p, 1, 2, 64, 64, 20, 32, 8) == 0
+    assert L.ec_cache_track_order(C.byref(fixed), order) == 4        # the fixed budget needs no list
+
+
 def test_a_zeroed_or_damaged_cache_struct_is_an_error_not_a_crash(L):
     """The struct is caller-owned plain data: every call that reads one re-checks it."""
     p = 0x10000

@@ -705,13 +705,63 @@ def test_cache_concat_restores_queue_order(N, H, D, C, len0, offset, steps, Tq):
     np.testing.assert_array_equal(host_bits(V_all.t), want_V)
 
 
-def test_cache_concat_rejects_the_ratio_policy_and_bad_shapes():
+@pytest.mark.parametrize("N,H,D,T,ratio,offset,steps,Tq", [
+    (2, 3, 128, 60, 0.5, 8, 45, 17),      # alternates between growing and evicting
+    (1, 4, 64, 100, 0.3, 25, 90, 40),     # the paper's recent distance; mostly evicts
+    (1, 2, 128, 40, 1.0, 4, 30, 5),       # ratio 1: never evicts, slots stay in order
+    (1, 2, 64, 3000, 0.4, 16, 700, 3),    # more rows than one slot list per launch holds (896)
+])
+def test_cache_concat_on_a_retention_ratio_cache(N, H, D, T, ratio, offset, steps, Tq):
+    """Sec. 3.1 (the instruction stage takes in the chat history) on top of Sec. 3.3's literal generation
+    rule: after a chain of grow / evict steps the physical slots are in no simple order; the tracked
+    queue order must reproduce the oracle's queue, oldest first, bit for bit, followed by the new rows."""
+    rng = np.random.default_rng(T + steps)
+    scale = 1.0 / math.sqrt(D)
+    len0 = orc.keep_count(T, ratio)
+    cap = len0 + steps
+    K0b, V0b = rand_bits(rng, (N, H, len0, D)), rand_bits(rng, (N, H, len0, D))
+    queue = orc.DecodeQueue(wl.bf16_bits_to_f64(K0b), wl.bf16_bits_to_f64(V0b), cap=cap + 1, n_seen=T)
+    Kc = torch.zeros((N, H, cap, D), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    Kc[:, :, :len0], Vc[:, :, :len0] = dev_bf16(K0b), dev_bf16(V0b)
+    cache = ec.ec_cache_init_ratio(Kc, Vc, len0, offset, ratio, T)
+    ws = scratch(ec.ec_decode_workspace(cache))
+    qb, kb, vb = (rand_bits(rng, (steps, N, H, D)) for _ in range(3))
+    for s in range(steps):
+        queue.step(qb[s], kb[s], vb[s], scale, policy=orc.POLICY_RATIO, offset=offset, ratio=ratio)
+    out = torch.empty((steps, N, H, D), dtype=torch.bfloat16, device="cuda")
+    ec.ec_decode_steps(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), cache, scale, out, ws)
+    P = cache.len
+    assert P == queue.len
+    order = [cache.queue_slots_host[j] for j in range(P)]
+    assert sorted(order) == list(range(P)) if ratio == 1.0 else len(set(order)) == P
+    Knb, Vnb = rand_bits(rng, (N, H, Tq, D)), rand_bits(rng, (N, H, Tq, D))
+    K_all = Guarded((N, H, P + Tq, D), torch.bfloat16, fill=float("nan"))
+    V_all = Guarded((N, H, P + Tq, D), torch.bfloat16, fill=float("nan"))
+    ec.ec_cache_concat(cache, dev_bf16(Knb), dev_bf16(Vnb), K_all.t, V_all.t)
+    K_all.check("K_all")
+    V_all.check("V_all")
+    want_K = np.concatenate([orc.round_bf16(queue.K[:, :P].reshape(N, H, P, D)), Knb], 2)
+    want_V = np.concatenate([orc.round_bf16(queue.V[:, :P].reshape(N, H, P, D)), Vnb], 2)
+    np.testing.assert_array_equal(host_bits(K_all.t), want_K)
+    np.testing.assert_array_equal(host_bits(V_all.t), want_V)
+    # the history feeds the importance of the new instruction exactly as a fixed-budget cache's does
+    Qnb = rand_bits(rng, (N, H, Tq, D))
+    scores = torch.empty((N, H, P + Tq), dtype=torch.float32, device="cuda")
+    ws_i = scratch(ec.ec_importance_workspace(N, H, Tq, D))
+    ec.ec_importance_prefix(dev_bf16(Qnb), K_all.t, scores, None, scale, ws_i)
+    assert ec.ec_device_status(ws_i) == ec.EC_OK
+    o_scores, _ = orc.importance_prefix(Qnb, want_K, scale)
+    assert_rel_close(scores, o_scores, SCORE_RTOL, what="importance over the ratio cache's history")
+
+
+def test_cache_concat_rejects_an_untracked_ratio_cache_and_bad_shapes():
     N, H, D, C = 1, 2, 64, 16
     Kc = torch.zeros((N, H, C + 8, D), dtype=torch.bfloat16, device="cuda")
     Vc = torch.zeros_like(Kc)
     new = torch.zeros((N, H, 4, D), dtype=torch.bfloat16, device="cuda")
     all_ = torch.zeros((N, H, C + 4, D), dtype=torch.bfloat16, device="cuda")
-    ratio_cache = ec.ec_cache_init_ratio(Kc, Vc, C, 4, 0.5, 32)
+    ratio_cache = ec.ec_cache_init_ratio(Kc, Vc, C, 4, 0.5, 32, track_order=False)
     with pytest.raises(ec.EcError) as e:
         ec.ec_cache_concat(ratio_cache, new, new, all_, all_.clone())
     assert e.value.status == ec.EC_ERR_ARG
