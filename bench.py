@@ -265,6 +265,7 @@ def whole_job_tokens_per_s(w: wl.Workload, world: int, ms_per_pass: float) -> fl
 def stage_figures(w: wl.Workload, C: int, imp_ms: float, mrg_ms: float, dec_ms: float, peaks: dict):
     """Algorithmic work of the three stages of one pass and the rates the measured times give."""
     units, T, D, S = w.N * w.heads, w.prompt_len, w.head_dim, w.decode_steps
+    w_ratio = w.keep_ratio
     # one decode launch: every cached K and V row once, q/k_new/v_new in, out and the overwritten slot out
     dec_bytes = units * (2 * C * D * 2 + 3 * D * 2 + D * 2 + 2 * D * 2)
     dec_gbs = dec_bytes / (dec_ms * 1e-3 / S) / 1e9
@@ -284,6 +285,10 @@ def stage_figures(w: wl.Workload, C: int, imp_ms: float, mrg_ms: float, dec_ms: 
     dec["bytes_per_launch"] = dec_bytes
     mrg = hbm(mrg_gbs)
     mrg["bytes_per_call"] = mrg_bytes
+    mixed, w = mixed_peak_for(peaks, w_ratio)
+    mrg["frac_of_mixed_stream"] = (mrg_gbs / mixed) if mixed else None
+    mrg["mixed_stream_peak"] = mixed
+    mrg["mixed_stream_write_every"] = w
     imp = {"achieved": imp_tflops, "unit": "TFLOP/s", "frac": imp_tflops / peaks["bf16_tflops"],
            "flops_per_call": imp_flops}
     return dec, mrg, imp
@@ -325,13 +330,20 @@ class DevicePass:
         if events is not None:
             events[3].record(self.stream)
 
-    def timed(self, warmup: int, steps: int, barrier, sampler):
-        """`warmup` untimed passes, then `steps` timed ones: whole time from one event pair around all of
-        them, stage times as means of per-pass event pairs. Returns (ms_per_pass, imp, mrg, dec, clocks)."""
+    def timed(self, warmup: int, steps: int, barrier, sampler, min_ms: float = 0.0):
+        """`warmup` untimed passes, then `steps` timed ones (more when `min_ms` asks for a longer timed
+        region, so that the clock sampler sees it): whole time from one event pair around all of them,
+        stage times as means of per-pass event pairs. Returns (ms_per_pass, imp, mrg, dec, clocks, steps)."""
         import torch
-        for _ in range(warmup):
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(warmup):
+            if i == warmup - 1:
+                w0.record(self.stream)
             self.run()
+        w1.record(self.stream)
         barrier()
+        if min_ms > 0.0 and warmup > 0:
+            steps = max(steps, int(np.ceil(min_ms / max(w0.elapsed_time(w1), 1e-3))))
         if sampler is not None:
             sampler.start()
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
@@ -349,7 +361,7 @@ class DevicePass:
         return (t_begin.elapsed_time(t_end) / steps,
                 float(np.mean([e[0].elapsed_time(e[1]) for e in ev])),
                 float(np.mean([e[1].elapsed_time(e[2]) for e in ev])),
-                float(np.mean([e[2].elapsed_time(e[3]) for e in ev])), clocks)
+                float(np.mean([e[2].elapsed_time(e[3]) for e in ev])), clocks, steps)
 
 
 def host_inputs(w: wl.Workload, pin: bool, threads: int):
@@ -358,33 +370,52 @@ def host_inputs(w: wl.Workload, pin: bool, threads: int):
     return tuple(bits_to_tensor(x, pin) for x in (Qb, Kb, Vb, qb, kb, vb))
 
 
-def read_stream_peak(ec, nbytes: int = 4 << 30, reps: int = 5):
-    """Read-only bandwidth of this GPU, measured here and now: best of `reps` passes of a 16-byte-load
-    sum kernel over a 4 GiB buffer (far above the L2), CUDA-event timed."""
+def stream_peaks(ec, nbytes: int = 4 << 30, reps: int = 5):
+    """Streaming rates of this GPU, measured here and now with the library's probe kernel over a 4 GiB
+    buffer (far above the L2), best of `reps`, CUDA-event timed: read-only, and reads with one 256-byte
+    row in 2 / 4 / 10 written back (the mixes of a merge at keep ratio 0.5 / 0.25 / 0.1; bytes counted
+    are reads + writes). Returns {"read_gbs": ..., "mixed_gbs": {2: ..., 4: ..., 10: ...}}."""
     import torch
     buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     buf.zero_()
+    dst = torch.empty(nbytes // 2, dtype=torch.uint8, device="cuda")
     sink = torch.zeros(1, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
-    ec.ec_probe_read_stream(buf, sink)
-    torch.cuda.synchronize()
-    best = None
-    for _ in range(reps):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        ec.ec_probe_read_stream(buf, sink)
-        b.record(stream)
+
+    def best_of(w):
+        run = (lambda: ec.ec_probe_read_stream(buf, sink)) if w == 0 else (lambda: ec.ec_probe_mixed_stream(buf, dst, w, sink))
+        run()
         torch.cuda.synchronize()
-        ms = a.elapsed_time(b)
-        best = ms if best is None else min(best, ms)
-    del buf
+        best = None
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            run()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b)
+            best = ms if best is None else min(best, ms)
+        moved = nbytes + (nbytes // w if w else 0)
+        return moved / (best * 1e-3) / 1e9
+
+    out = {"read_gbs": best_of(0), "mixed_gbs": {w: best_of(w) for w in (2, 4, 10)}}
+    del buf, dst
     torch.cuda.empty_cache()
-    return nbytes / (best * 1e-3) / 1e9
+    return out
+
+
+def mixed_peak_for(peaks: dict, keep_ratio: float):
+    """The measured mixed-stream rate whose write share is nearest to a merge at this keep ratio."""
+    mixed = peaks.get("mixed_gbs")
+    if not mixed:
+        return None, None
+    w = min(mixed, key=lambda k: abs(1.0 / k - keep_ratio))
+    return mixed[w], w
 
 
 def measure_other_workloads(ec, peaks, threads: int, passes: int, local: int):
     """The remaining configurations, each timed like the headline (same calls, same event placement)
-    with 3 warm-up and `passes` timed passes; every keep ratio of a sweep is its own entry."""
+    with 3 warm-up and at least `passes` timed passes (at least 0.4 s of them); every keep ratio of a sweep is its own entry."""
     import dataclasses
     import gc
     import torch
@@ -397,11 +428,12 @@ def measure_other_workloads(ec, peaks, threads: int, passes: int, local: int):
             w = dataclasses.replace(base, keep_ratios=(ratio,))
             dp = DevicePass(w, host=host) if first is None else DevicePass(w, resident=first)
             first = first or dp
-            ms, imp_ms, mrg_ms, dec_ms, clocks = dp.timed(3, passes, torch.cuda.synchronize, ClockSampler(local))
+            ms, imp_ms, mrg_ms, dec_ms, clocks, done = dp.timed(3, passes, torch.cuda.synchronize, ClockSampler(local),
+                                                                min_ms=400.0)
             dec, mrg, imp = stage_figures(w, dp.C, imp_ms, mrg_ms, dec_ms, peaks)
             key = name if len(base.keep_ratios) == 1 else f"{name}@{ratio:g}"
             result[key] = {
-                "config": workload_config(w, dp.C), "passes": passes, "ms_per_pass": ms,
+                "config": workload_config(w, dp.C), "passes": done, "ms_per_pass": ms,
                 "tokens_per_s": w.batch * w.decode_steps / (ms * 1e-3),
                 "stages_ms": {"importance": imp_ms, "select_merge": mrg_ms, "decode_loop": dec_ms,
                               "decode_per_token_us": dec_ms * 1e3 / w.decode_steps},
@@ -454,8 +486,8 @@ def run_ours(args, w: wl.Workload):
             dist.barrier()
             torch.cuda.synchronize()
 
-    total_ms, imp_ms, mrg_ms, dec_ms, clocks = dp.timed(args.warmup, args.steps, barrier,
-                                                        ClockSampler(local) if rank == 0 else None)
+    total_ms, imp_ms, mrg_ms, dec_ms, clocks, _ = dp.timed(args.warmup, args.steps, barrier,
+                                                           ClockSampler(local) if rank == 0 else None)
     ms_per_step = total_ms
     splits = ec.ec_decode_splits(dp.sess.cache)
 
@@ -534,7 +566,7 @@ def run_ours(args, w: wl.Workload):
 
     peaks = measured_peaks()
     if world == 1 and not args.no_read_peak:
-        peaks["read_gbs"] = read_stream_peak(ec)
+        peaks.update(stream_peaks(ec))
     tokens = w.batch * S * world
     value = whole_job_tokens_per_s(w, world, ms_per_step)
     dec, mrg, imp = stage_figures(w, C, imp_ms, mrg_ms, dec_ms, peaks)
@@ -543,7 +575,7 @@ def run_ours(args, w: wl.Workload):
 
     roofline = {"kernel": "decode_kernel", "bound": "hbm", "achieved": dec["achieved"], "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": dec["frac"], "peak_source": peaks["source"] + " (copy: half reads, half writes)",
-                "read_stream_peak": peaks.get("read_gbs"), "frac_of_read_stream": dec["frac_of_read_stream"],
+                "read_stream_peak": peaks.get("read_gbs"), "mixed_stream_peaks": peaks.get("mixed_gbs"), "frac_of_read_stream": dec["frac_of_read_stream"],
                 "frac_of_nominal_8TBs": dec["frac_of_nominal_8TBs"], "bytes_per_launch": dec["bytes_per_launch"],
                 "decode_splits": splits, "traffic": decode_traffic(w.name),
                 "note": ("algorithmic bytes of one step / (decode loop time / steps); consecutive steps of the "

@@ -398,6 +398,16 @@ int ec_cache_concat(const ec_cache *c, const void *K_new_dev, const void *V_new_
 int ec_probe_read_stream(const void *buf_dev, size_t bytes, unsigned *sink_dev, void *stream);
 
 /*
+ * (No counterpart in the paper.) The same stream with writes mixed in: of every `write_every`
+ * consecutive 256-byte rows read, one is also written to dst_dev, packed densely, which is the
+ * read/write mix of the merge kernel at keep ratio 1/write_every (write_every = 0: no writes).
+ * Timing it gives the ceiling for that mix on this GPU.
+ *   dst_dev   device, 16-byte aligned, at least ceil(bytes/256 / write_every) * 256 bytes
+ */
+int ec_probe_mixed_stream(const void *buf_dev, size_t bytes, void *dst_dev, int write_every, unsigned *sink_dev,
+                          void *stream);
+
+/*
  * How many CTAs would share one unit's rows if ec_decode_step were called on *c now (1: one
  * CTA per unit, the layout of large batches; > 1: the split path with in-kernel merge).
  * 0 when *c is invalid.

@@ -28,7 +28,7 @@ EXPORTS = (
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
     "ec_cache_init", "ec_cache_init_ratio", "ec_cache_track_order", "ec_cache_concat", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc", "ec_compress_host", "ec_decode_steps_host",
-    "ec_probe_read_stream", "ec_decode_splits",
+    "ec_probe_read_stream", "ec_probe_mixed_stream", "ec_decode_splits",
 )
 
 
@@ -113,6 +113,8 @@ def lib() -> C.CDLL:
     L.ec_decode_step_noalloc.argtypes = [vp, vp, vp, C.POINTER(ec_cache), f, vp, C.POINTER(i), C.POINTER(i), vp]
     L.ec_probe_read_stream.restype = i
     L.ec_probe_read_stream.argtypes = [vp, sz, vp, vp]
+    L.ec_probe_mixed_stream.restype = i
+    L.ec_probe_mixed_stream.argtypes = [vp, sz, vp, i, vp, vp]
     L.ec_decode_splits.restype = i
     L.ec_decode_splits.argtypes = [C.POINTER(ec_cache)]
     _lib = L
@@ -355,6 +357,15 @@ def ec_probe_read_stream(buf: torch.Tensor, sink: torch.Tensor) -> None:
     """Enqueue one read-only pass over `buf` (any dtype, byte size a multiple of 16); `sink`: uint32/int32 [1]."""
     _check(lib().ec_probe_read_stream(_ptr(buf), buf.numel() * buf.element_size(), _ptr(sink), _stream()),
            "ec_probe_read_stream")
+
+
+def ec_probe_mixed_stream(buf: torch.Tensor, dst: torch.Tensor, write_every: int, sink: torch.Tensor) -> None:
+    """ec_probe_read_stream that also writes one 256-byte row in `write_every` to `dst` (densely)."""
+    need = -(-(buf.numel() * buf.element_size() // 256) // max(1, write_every)) * 256
+    if write_every > 0 and dst.numel() * dst.element_size() < need:
+        raise ValueError("dst is too small for this write ratio")
+    _check(lib().ec_probe_mixed_stream(_ptr(buf), buf.numel() * buf.element_size(), _ptr(dst), int(write_every),
+                                       _ptr(sink), _stream()), "ec_probe_mixed_stream")
 
 
 def ec_decode_splits(cache: ec_cache) -> int:

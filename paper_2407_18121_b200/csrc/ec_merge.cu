@@ -22,6 +22,9 @@ namespace {
 #ifndef EC_MERGE_UNROLL
 #define EC_MERGE_UNROLL 8
 #endif
+#ifndef EC_MERGE_MIN_CTAS
+#define EC_MERGE_MIN_CTAS 1
+#endif
 constexpr int kMergeThreads = EC_MERGE_THREADS;
 constexpr int kRowsPerCta = EC_MERGE_ROWS_PER_CTA;
 constexpr int kUnroll = EC_MERGE_UNROLL;
@@ -50,7 +53,7 @@ __device__ __forceinline__ int first_bucket_from(const int32_t *anch, int C, int
 // halves see the same bucket boundaries (for D = 128 a group is exactly one warp: no divergence).
 // grid.x = units * slices (equal slices of at most 256 rows). Dynamic shared memory: the unit's C anchors.
 template <int LPR>
-__global__ void __launch_bounds__(kMergeThreads)
+__global__ void __launch_bounds__(kMergeThreads, EC_MERGE_MIN_CTAS)
 merge_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, const int32_t *__restrict__ anchor_pos,
              int T, int C, int slices, uint4 *__restrict__ Kc, uint4 *__restrict__ Vc, int cap)
 {
