@@ -10,11 +10,15 @@
 // row in pass 2 and every reduction stays inside a thread (no atomics, run-to-run identical).
 //
 // A work item is a "stationary" 128-row tile of one unit, past which the other operand's
-// tiles are streamed. CTAs are persistent (two per SM): each walks a fixed list of item
-// pairs (a heavy tile and its light complement, so that pairs cost about the same) and
-// keeps its barriers, TMEM allocation and TMA ring alive across items. Warp roles: warp 0
-// issues TMA loads, warp 1 issues MMAs and owns the TMEM allocation, warps 2..5 (one thread
-// per TMEM lane) do the softmax arithmetic.
+// tiles are streamed. CTAs are persistent (two per SM) and keep their barriers, TMEM
+// allocation and TMA ring alive across items. Items are handed out in order (units in order
+// for L2 reuse, a unit's tiles from the longest to the shortest) from a counter in global
+// memory: a CTA's first item is its block index, every later one comes from an atomic
+// increment that the TMA thread issues one item ahead and publishes to the other roles
+// through a small ring in shared memory. Which CTA takes which item does not affect any
+// result. Warp roles: warp 0 issues TMA loads (and L2 prefetches for the item after the
+// current one), warp 1 issues MMAs and owns the TMEM allocation, warps 2..9 (two threads per
+// TMEM lane) do the softmax arithmetic.
 // Every mbarrier wait is bounded in time; on expiry the CTA records a status word and leaves.
 #include "ec_common.cuh"
 
@@ -29,6 +33,7 @@ constexpr int kTileRows = 128;            // rows of a tile = MMA M = MMA N
 constexpr int kThreads = 320;             // 10 warps: TMA, MMA, 8 x softmax (two per TMEM lane quarter)
 constexpr int kAccBufs = 2;               // TMEM accumulator buffers (128 columns each)
 constexpr int kTmemCols = 256;
+constexpr int kSched = 4;                 // slots of the ring that publishes item numbers to the roles
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s per wait, then give up
@@ -199,11 +204,12 @@ struct Smem {
     static constexpr int kComb = kLse + kAccBufs * kTileRows * 4;         // 128 x float2: half-row results
     static constexpr int kBars = kComb + kTileRows * 8;
     // barrier slots (8 bytes each): stat_full, stat_empty, full[STAGES], empty[STAGES],
-    // acc_full[2], acc_empty[2], lse_ready[2], comb_full, comb_empty
-    static constexpr int kNumBars = 2 + 2 * STAGES + 3 * kAccBufs + 2;
+    // acc_full[2], acc_empty[2], lse_ready[2], comb_full, comb_empty, sched_full[kSched], sched_empty[kSched]
+    static constexpr int kNumBars = 2 + 2 * STAGES + 3 * kAccBufs + 2 + 2 * kSched;
     static constexpr int kTmemSlot = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemSlot + 4;
-    static constexpr int kTotal = kAbort + 4;
+    static constexpr int kSchedItems = (kAbort + 4 + 15) & ~15;           // kSched published items (int4 each)
+    static constexpr int kTotal = kSchedItems + kSched * 16;
     static constexpr int kDynBytes = kTotal + 1024;                       // slack for 1024-byte alignment
 };
 
@@ -240,8 +246,9 @@ constexpr int kPass1 = 0, kPass2Sum = 1, kPass2Max = 2;
 template <int D, int STAGES, int MODE>
 __global__ void __launch_bounds__(kThreads, 2)
 importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const Geometry geo, const Fold fold, int n_super, float c, float *__restrict__ lse2,
-                  float *__restrict__ lse_out, float *__restrict__ scores, int *__restrict__ status)
+                  const Geometry geo, const Fold fold, int n_items, int tail_units, float c, float *__restrict__ lse2,
+                  float *__restrict__ lse_out, float *__restrict__ scores, int *__restrict__ status,
+                  int *__restrict__ next_item)
 {
     constexpr bool PASS2 = MODE != kPass1;
     constexpr bool TAKE_MAX = MODE == kPass2Max;
@@ -263,6 +270,9 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     auto bar_lse = [&](int b) { return bars + 8u * (2 + 2 * STAGES + 2 * kAccBufs + b); };
     const uint32_t bar_comb_full = bars + 8u * (2 + 2 * STAGES + 3 * kAccBufs);
     const uint32_t bar_comb_empty = bar_comb_full + 8u;
+    auto bar_sched_full = [&](uint32_t k) { return bar_comb_empty + 8u * (1 + k); };
+    auto bar_sched_empty = [&](uint32_t k) { return bar_comb_empty + 8u * (1 + kSched + k); };
+    int4 *sched_s = reinterpret_cast<int4 *>(base_ptr + L::kSchedItems);   // {unit, stationary tile, first streamed tile, count}
     float2 *comb_s = reinterpret_cast<float2 *>(base_ptr + L::kComb);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + L::kTmemSlot);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + L::kAbort);
@@ -272,26 +282,12 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const CUtensorMap *map_stat = PASS2 ? &map_k : &map_q;
     const CUtensorMap *map_strm = PASS2 ? &map_q : &map_k;
     const int nts = PASS2 ? geo.ntk : geo.ntq;              // stationary tiles per unit
-    const int spu = (nts + 1) / 2;                          // item pairs per unit
-
-    // Static schedule: in round k this CTA takes pair k*grid + (cta + k*rot) mod grid, so that a round
-    // covers consecutive pairs (units in order, for L2 reuse). With an odd tile count the unit's
-    // middle tile is a pair of half the cost, and a CTA meets cost classes cta + k*(grid + rot) mod
-    // spu: when grid mod spu shares a factor with spu, some CTAs would never get a cheap pair
-    // (measured: 15% slower at T = 320, 10% at T = 896), so rot then makes (grid + rot) mod spu = 1.
-    // Otherwise rot = 0. Only the last round can be partial.
     const int grid_n = (int)gridDim.x;
-    int rot = 0;
-    if ((nts & 1) && spu > 1) {
-        int a = grid_n % spu, b = spu;
-        while (a) { const int t = b % a; b = a; a = t; }      // b = gcd(grid mod spu, spu)
-        if (b != 1) rot = ((1 - grid_n) % spu + spu) % spu;
-    }
-    auto pair_of_round = [&](int k) -> int {
-        const long long sidx = (long long)k * grid_n + ((int)blockIdx.x + k * rot) % grid_n;
-        return sidx < n_super ? (int)sidx : -1;
-    };
 
+    if (threadIdx.x == 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+    }
     // a CTA of this launch has already given up: leave at once instead of timing out again
     if (threadIdx.x == 0) *abort_flag = *reinterpret_cast<volatile int *>(status);
     __syncthreads();
@@ -308,6 +304,10 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
         mbar_init(bar_comb_full, 4 * 32);
         mbar_init(bar_comb_empty, 4 * 32);
+        for (uint32_t k = 0; k < (uint32_t)kSched; ++k) {
+            mbar_init(bar_sched_full(k), 1);
+            mbar_init(bar_sched_empty(k), 1 + 8);           // the MMA thread and one lane of each softmax warp
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -321,21 +321,30 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // Every role walks the same item list with the same counters: `it` counts items (stationary
-    // tiles), `tg` counts streamed tiles; ring slots and barrier phases derive from them.
+    // Every role walks the same sequence of items with the same counters: `it` counts items
+    // (stationary tiles), `tg` counts streamed tiles; ring slots and barrier phases derive from them.
     uint32_t it = 0, tg = 0;
     bool alive = true;
 
-    // item `sub` (0 = heavy, 1 = its complement) of pair `sidx`: stationary tile and streamed range
-    auto item_of = [&](int sidx, int sub, int &unit, int &st, int &first, int &count) -> bool {
-        unit = sidx / spu;
-        const int pi = sidx - unit * spu;
-        const int heavy = PASS2 ? pi : nts - 1 - pi, light = nts - 1 - heavy;
-        if (sub == 1 && light == heavy) return false;
-        st = sub ? light : heavy;
+    // item -> unit, stationary tile, first streamed tile and number of streamed tiles. Units go in
+    // order and a unit's items from the longest to the shortest, except for the last `tail_units`
+    // units, which are taken together: all their longest items first, their shortest last. The work
+    // handed out last is then made of short items of a few units (longest-first list scheduling),
+    // and those units' tensors still fit the L2 together.
+    const int n_units = n_items / nts, head_items = (n_units - tail_units) * nts;
+    auto decode_item = [&](int item, int &unit, int &st, int &first, int &count) {
+        int k;
+        if (item < head_items) {
+            unit = item / nts;
+            k = item - unit * nts;
+        } else {
+            const int j = item - head_items;
+            k = j / tail_units;
+            unit = (n_units - tail_units) + (j - k * tail_units);
+        }
+        st = PASS2 ? k : nts - 1 - k;
         if (PASS2) { first = geo.imin(st); count = geo.ntq - first; }
         else       { first = geo.jmax(st); count = first + 1; }
-        return true;
     };
     auto stream_tile = [&](int first, int t) { return PASS2 ? first + t : first - t; };
 
@@ -343,33 +352,40 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t armed = 0, stat_armed = 0;           // streamed tiles / stationary tiles whose copies were started
-            for (int round = 0, sidx; alive && (sidx = pair_of_round(round)) >= 0; ++round) {
-                for (int sub = 0; alive && sub < 2; ++sub) {
-                    int unit, st, first, count;
-                    if (!item_of(sidx, sub, unit, st, first, count)) break;
-                    // The item's first streamed tile goes out first: its ring stage was released by an
-                    // earlier MMA of the previous item, whereas the stationary buffer is free only once
-                    // that item's last MMA has completed.
-                    for (int t = 0; t < count; ++t, ++tg) {
-                        const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
-                        if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                        mbar_expect_tx(bar_full(s), kTileBytes);
+            int item = (int)blockIdx.x;                   // the first item needs no counter: one per CTA
+            for (uint32_t k = 0; alive; ++k) {
+                const uint32_t sl = k % kSched, sph = (k / kSched) & 1u;
+                if (!mbar_wait(bar_sched_empty(sl), sph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                int unit = -1, st = 0, first = 0, count = 0;  // unit -1: no work left, every role leaves
+                if (item < n_items) decode_item(item, unit, st, first, count);
+                sched_s[sl] = make_int4(unit, st, first, count);
+                mbar_arrive(bar_sched_full(sl));
+                if (unit < 0) break;
+                // the item after this one: asked for now, needed only when this item's copies are under way
+                const int next = grid_n + atomicAdd(next_item, 1);
+                // The item's first streamed tile goes out first: its ring stage was released by an
+                // earlier MMA of the previous item, whereas the stationary buffer is free only once
+                // that item's last MMA has completed.
+                for (int t = 0; t < count; ++t, ++tg) {
+                    const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
+                    if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    mbar_expect_tx(bar_full(s), kTileBytes);
+#pragma unroll
+                    for (int bx = 0; bx < kBoxes; ++bx)
+                        tma_load_3d(base + L::kStage0 + s * kTileBytes + bx * kBoxBytes, map_strm, bx * 64,
+                                    stream_tile(first, t) * kTileRows, unit, bar_full(s));
+                    armed = tg + 1;
+                    if (t == 0) {
+                        if (!mbar_wait(bar_stat_empty, (it + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                        mbar_expect_tx(bar_stat_full, kTileBytes);
 #pragma unroll
                         for (int bx = 0; bx < kBoxes; ++bx)
-                            tma_load_3d(base + L::kStage0 + s * kTileBytes + bx * kBoxBytes, map_strm, bx * 64,
-                                        stream_tile(first, t) * kTileRows, unit, bar_full(s));
-                        armed = tg + 1;
-                        if (t == 0) {
-                            if (!mbar_wait(bar_stat_empty, (it + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                            mbar_expect_tx(bar_stat_full, kTileBytes);
-#pragma unroll
-                            for (int bx = 0; bx < kBoxes; ++bx)
-                                tma_load_3d(base + L::kStat + bx * kBoxBytes, map_stat, bx * 64, st * kTileRows, unit, bar_stat_full);
-                            stat_armed = it + 1;
-                        }
+                            tma_load_3d(base + L::kStat + bx * kBoxBytes, map_stat, bx * 64, st * kTileRows, unit, bar_stat_full);
+                        stat_armed = it + 1;
                     }
-                    ++it;
                 }
+                ++it;
+                item = next;
             }
             if (*abort_flag) {
                 // let copies that are still in flight land before the CTA gives its memory back
@@ -381,30 +397,32 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            for (int round = 0, sidx; alive && (sidx = pair_of_round(round)) >= 0; ++round) {
-                for (int sub = 0; alive && sub < 2; ++sub) {
-                    int unit, st, first, count;
-                    if (!item_of(sidx, sub, unit, st, first, count)) break;
-                    if (!mbar_wait(bar_stat_full, it & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                    for (int t = 0; t < count; ++t, ++tg) {
-                        const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
-                        const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
-                        if (!mbar_wait(bar_acc_empty(b), bph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                        if (!mbar_wait(bar_full(s), ph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                        tc_fence_after();
-                        const uint32_t a0 = base + L::kStat, b0 = base + L::kStage0 + s * kTileBytes;
+            for (uint32_t k = 0; alive; ++k) {
+                const uint32_t sl = k % kSched, sph = (k / kSched) & 1u;
+                if (!mbar_wait(bar_sched_full(sl), sph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                const int4 d = sched_s[sl];
+                mbar_arrive(bar_sched_empty(sl));
+                if (d.x < 0) break;
+                const int count = d.w;
+                if (!mbar_wait(bar_stat_full, it & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                for (int t = 0; t < count; ++t, ++tg) {
+                    const uint32_t s = tg % STAGES, ph = (tg / STAGES) & 1u;
+                    const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
+                    if (!mbar_wait(bar_acc_empty(b), bph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    if (!mbar_wait(bar_full(s), ph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t a0 = base + L::kStat, b0 = base + L::kStage0 + s * kTileBytes;
 #pragma unroll
-                        for (int k = 0; k < D / 16; ++k) {
-                            const uint32_t off = (uint32_t)(k / 4) * kBoxBytes + (uint32_t)(k % 4) * 32u;
-                            umma_bf16(tmem_base + b * kTileRows, umma_desc(a0 + off), umma_desc(b0 + off), kIdesc,
-                                      k > 0 ? 1u : 0u);
-                        }
-                        umma_commit(bar_empty(s));       // stage reusable once these MMAs have read it
-                        umma_commit(bar_acc_full(b));    // accumulator ready for the softmax warps
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (uint32_t)(kk / 4) * kBoxBytes + (uint32_t)(kk % 4) * 32u;
+                        umma_bf16(tmem_base + b * kTileRows, umma_desc(a0 + off), umma_desc(b0 + off), kIdesc,
+                                  kk > 0 ? 1u : 0u);
                     }
-                    if (alive) umma_commit(bar_stat_empty);   // stationary tile no longer read
-                    ++it;
+                    umma_commit(bar_empty(s));       // stage reusable once these MMAs have read it
+                    umma_commit(bar_acc_full(b));    // accumulator ready for the softmax warps
                 }
+                if (alive) umma_commit(bar_stat_empty);   // stationary tile no longer read
+                ++it;
             }
         }
     } else {
@@ -417,165 +435,185 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int r = q4 * 32 + lane;                         // row of the stationary tile = TMEM lane
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(half * 64);
         const int Tk = geo.Tk();
-        for (int round = 0, sidx; alive && (sidx = pair_of_round(round)) >= 0; ++round) {
-            for (int sub = 0; alive && sub < 2; ++sub) {
-                int unit, st, first, count;
-                if (!item_of(sidx, sub, unit, st, first, count)) break;
-                const size_t lse_row = (size_t)unit * geo.ntq * kTileRows;
-                float mrun = -INFINITY, Z = 0.f;                      // pass 1 running max / sum (log2 domain)
-                float2 accA = make_float2(0.f, 0.f), accB = accA;     // pass 2 column sum, four chains
-                float lse_ahead = 0.f;
-                if (PASS2 && half == 0) lse_ahead = lse2[lse_row + (size_t)first * kTileRows + r];
-                for (int t = 0; t < count; ++t, ++tg) {
-                    const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
-                    const int tile = stream_tile(first, t);
-                    // off = 128*(query tile - key tile) + P: element (row, col) is visible iff
-                    //   pass 1 (row = query, col = key):  col <= row + off
-                    //   pass 2 (row = key,  col = query): col >= row - off
-                    const int off = (PASS2 ? tile - st : st - tile) * kTileRows + geo.P;
-                    const bool masked = off < kTileRows - 1;
-                    if (PASS2) {
-                        // the first-half threads stage one entry each of the tile's lse (fetched one tile
-                        // ahead, so its latency hides behind the previous tile's math), then all wait
-                        // (bounded) for the 128 entries. Every softmax thread, readers of the second half
-                        // included, arrives on the tile's barrier: a thread that has passed the rendezvous
-                        // of tile t+1 therefore knows that all 256 have finished reading tile t's entries,
-                        // and only then may buffer b be overwritten for tile t+2.
-                        if (half == 0) {
-                            lse_s[b * kTileRows + r] = -lse_ahead;    // staged negated: exponent = v*c + (-lse)
-                            mbar_arrive(bar_lse(b));
-                            if (t + 1 < count)
-                                lse_ahead = lse2[lse_row + (size_t)stream_tile(first, t + 1) * kTileRows + r];
-                        } else {
-                            mbar_arrive(bar_lse(b));
-                        }
-                        if (!mbar_wait(bar_lse(b), bph, abort_flag, status)) { alive = false; break; }
-                    }
-                    if (!mbar_wait(bar_acc_full(b), bph, abort_flag, status)) { alive = false; break; }
-                    tc_fence_after();
-
-                    // `ch` = index of the 32-column chunk inside the 128-column tile
-                    auto chunk = [&](uint32_t (&raw)[32], int ch, auto mask_tag) {
-                        constexpr bool MASKED = decltype(mask_tag)::value;
-                        float v[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]);
-                        if (!PASS2) {
-                            if constexpr (MASKED) {
-                                const int lim = r + off - ch * 32;            // columns i <= lim are visible
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) if (i > lim) v[i] = -INFINITY;
-                            }
-                            float cm4[4] = {v[0], v[1], v[2], v[3]};      // four chains instead of one of 31
-#pragma unroll
-                            for (int i = 4; i < 32; ++i) cm4[i & 3] = fmaxf(cm4[i & 3], v[i]);
-                            const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
-                            const float mnew = fmaxf(mrun, cm * c);
-                            if (mnew != -INFINITY) {
-                                float2 part[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                                sum_exp2(v, c, mnew, part);
-                                Z = Z * fast_exp2(mrun - mnew) + ((part[0].x + part[0].y) + (part[1].x + part[1].y));
-                                mrun = mnew;
-                            }
-                        } else {
-                            const float4 *ls = reinterpret_cast<const float4 *>(lse_s + b * kTileRows + ch * 32);
-                            const int lim = r - off - ch * 32;                // columns i >= lim are visible
-                            const float2 c2 = make_float2(c, c);
-#pragma unroll
-                            for (int i4 = 0; i4 < 8; ++i4) {
-                                const float4 nl = ls[i4];                     // -lse of four query rows
-                                const float2 a01 = __ffma2_rn(make_float2(v[i4 * 4 + 0], v[i4 * 4 + 1]), c2, make_float2(nl.x, nl.y));
-                                const float2 a23 = __ffma2_rn(make_float2(v[i4 * 4 + 2], v[i4 * 4 + 3]), c2, make_float2(nl.z, nl.w));
-                                const float2 e01 = exp2_pair(a01, i4 * 2), e23 = exp2_pair(a23, i4 * 2 + 1);
-                                float p0 = e01.x, p1 = e01.y, p2 = e23.x, p3 = e23.y;
-                                if constexpr (MASKED) {
-                                    if (i4 * 4 + 0 < lim) p0 = 0.f;
-                                    if (i4 * 4 + 1 < lim) p1 = 0.f;
-                                    if (i4 * 4 + 2 < lim) p2 = 0.f;
-                                    if (i4 * 4 + 3 < lim) p3 = 0.f;
-                                }
-                                if constexpr (TAKE_MAX) {
-                                    accA.x = fmaxf(accA.x, p0); accA.y = fmaxf(accA.y, p1);
-                                    accB.x = fmaxf(accB.x, p2); accB.y = fmaxf(accB.y, p3);
-                                } else {
-                                    accA = __fadd2_rn(accA, make_float2(p0, p1));
-                                    accB = __fadd2_rn(accB, make_float2(p2, p3));
-                                }
-                            }
-                        }
-                    };
-
-                    // Only tiles the diagonal crosses pay for the mask: they run a separate instance.
-                    auto tile_body = [&](auto mask_tag) {
-                        constexpr bool MASKED = decltype(mask_tag)::value;
-                        const uint32_t col0 = lane_addr + b * kTileRows;
-                        // A chunk the mask hides from all 32 rows of this warp is neither read nor
-                        // exponentiated (on a diagonal tile that is 6 of the 16 warp x chunk blocks).
-                        //   pass 1: column visible iff col <= row + off  -> hidden iff first col > last row + off
-                        //   pass 2: column visible iff col >= row - off  -> hidden iff last col < first row - off
-                        auto hidden = [&](int ch) {
-                            if (!MASKED) return false;
-                            return PASS2 ? (ch * 32 + 31 < q4 * 32 - off) : (ch * 32 > q4 * 32 + 31 + off);
-                        };
-                        const bool skip_a = hidden(half * 2), skip_b = hidden(half * 2 + 1);   // warp-uniform
-                        auto release = [&]() {
-                            tc_fence_before();               // all TMEM reads of this tile are done:
-                            __syncwarp();                    // hand the accumulator back before the last chunk's math
-                            if (lane == 0) mbar_arrive(bar_acc_empty(b));
-                        };
-                        if (!skip_a && !skip_b) {
-                            // this thread's 64 columns: the second 32 are in flight while the first are processed
-                            uint32_t ra[32], rb[32];
-                            tmem_ld32_async(col0, ra);
-                            tmem_ld_wait(ra);
-                            tmem_ld32_async(col0 + 32, rb);
-                            chunk(ra, half * 2, mask_tag);
-                            tmem_ld_wait(rb);
-                            release();
-                            chunk(rb, half * 2 + 1, mask_tag);
-                        } else if (skip_a && skip_b) {
-                            release();
-                        } else {
-                            const int which = skip_a ? 1 : 0;     // the one chunk some row of the warp can see
-                            uint32_t ra[32];
-                            tmem_ld32_async(col0 + 32 * which, ra);
-                            tmem_ld_wait(ra);
-                            release();
-                            chunk(ra, half * 2 + which, mask_tag);
-                        }
-                    };
-                    if (masked) tile_body(std::true_type{});
-                    else tile_body(std::false_type{});
-                }
-                if (!alive) break;
-
-                // the two halves of a row meet: the second-half thread hands its result over
-                const uint32_t iph = it & 1u;
-                const float own = TAKE_MAX ? fmaxf(fmaxf(accA.x, accA.y), fmaxf(accB.x, accB.y))
-                                           : (accA.x + accA.y) + (accB.x + accB.y);
-                if (half == 1) {
-                    if (!mbar_wait(bar_comb_empty, iph ^ 1u, abort_flag, status)) { alive = false; break; }
-                    comb_s[r] = PASS2 ? make_float2(own, 0.f) : make_float2(mrun, Z);
-                    mbar_arrive(bar_comb_full);
-                } else {
-                    if (!mbar_wait(bar_comb_full, iph, abort_flag, status)) { alive = false; break; }
-                    const float2 o = comb_s[r];
-                    mbar_arrive(bar_comb_empty);
-                    const int row = st * kTileRows + r;
-                    if (!PASS2) {
-                        const float M = fmaxf(mrun, o.x);             // finite: column 0 of some tile is visible
-                        const float Zs = Z * fast_exp2(mrun - M) + o.y * fast_exp2(o.x - M);
-                        const float l2 = (row < geo.Tq) ? M + __log2f(Zs) : INFINITY;
-                        lse2[lse_row + row] = l2 - (fold.wa + fold.wb * (float)(row - (geo.Tq - 1)));   // +inf stays +inf
-                        if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
-                    } else if (row < Tk) {
-                        float total = TAKE_MAX ? fmaxf(own, o.x) : own + o.x;
-                        if (fold.mean) total /= (float)(geo.Tq - (row > geo.P ? row - geo.P : 0));   // queries that see this key
-                        scores[(size_t)unit * Tk + row] = total;
-                    }
-                }
-                ++it;
+        // The next item's description is normally picked up while this item's last tile is worked on
+        // (the TMA thread publishes it ahead), and in pass 2 the load of its first lse entry starts
+        // then, so that the start of an item costs no round trip to shared or global memory.
+        int4 next_d = make_int4(-1, 0, 0, 0);
+        float lse_next = 0.f;
+        bool have_next = false;
+        for (uint32_t k = 0; alive; ++k) {
+            const uint32_t sl = k % kSched, sph = (k / kSched) & 1u;
+            if (!have_next) {
+                if (!mbar_wait(bar_sched_full(sl), sph, abort_flag, status)) { alive = false; break; }
+                next_d = sched_s[sl];
             }
+            const int unit = next_d.x, st = next_d.y, first = next_d.z, count = next_d.w;
+            __syncwarp();                                         // every lane has read the slot
+            if (lane == 0) mbar_arrive(bar_sched_empty(sl));
+            if (unit < 0) break;
+            const size_t lse_row = (size_t)unit * geo.ntq * kTileRows;
+            float mrun = -INFINITY, Z = 0.f;                      // pass 1 running max / sum (log2 domain)
+            float2 accA = make_float2(0.f, 0.f), accB = accA;     // pass 2 column sum, four chains
+            float lse_ahead = 0.f;
+            if (PASS2 && half == 0) lse_ahead = have_next ? lse_next : lse2[lse_row + (size_t)first * kTileRows + r];
+            have_next = false;
+            for (int t = 0; t < count; ++t, ++tg) {
+                const uint32_t b = tg % kAccBufs, bph = (tg / kAccBufs) & 1u;
+                const int tile = stream_tile(first, t);
+                if (t == count - 1) {
+                    // last tile: look (without waiting) whether the next item is published; the warp decides as one
+                    const uint32_t nsl = (k + 1u) % kSched, nph = ((k + 1u) / kSched) & 1u;
+                    have_next = __all_sync(0xffffffffu, mbar_try(bar_sched_full(nsl), nph));
+                    if (have_next) next_d = sched_s[nsl];
+                }
+                // off = 128*(query tile - key tile) + P: element (row, col) is visible iff
+                //   pass 1 (row = query, col = key):  col <= row + off
+                //   pass 2 (row = key,  col = query): col >= row - off
+                const int off = (PASS2 ? tile - st : st - tile) * kTileRows + geo.P;
+                const bool masked = off < kTileRows - 1;
+                if (PASS2) {
+                    // the first-half threads stage one entry each of the tile's lse (fetched one tile
+                    // ahead, so its latency hides behind the previous tile's math), then all wait
+                    // (bounded) for the 128 entries. Every softmax thread, readers of the second half
+                    // included, arrives on the tile's barrier: a thread that has passed the rendezvous
+                    // of tile t+1 therefore knows that all 256 have finished reading tile t's entries,
+                    // and only then may buffer b be overwritten for tile t+2.
+                    if (half == 0) {
+                        lse_s[b * kTileRows + r] = -lse_ahead;    // staged negated: exponent = v*c + (-lse)
+                        mbar_arrive(bar_lse(b));
+                        if (t + 1 < count)
+                            lse_ahead = lse2[lse_row + (size_t)stream_tile(first, t + 1) * kTileRows + r];
+                        else if (have_next && next_d.x >= 0)
+                            lse_next = lse2[((size_t)next_d.x * geo.ntq + (size_t)next_d.z) * kTileRows + r];
+                    } else {
+                        mbar_arrive(bar_lse(b));
+                    }
+                    if (!mbar_wait(bar_lse(b), bph, abort_flag, status)) { alive = false; break; }
+                }
+                if (!mbar_wait(bar_acc_full(b), bph, abort_flag, status)) { alive = false; break; }
+                tc_fence_after();
+
+                // `ch` = index of the 32-column chunk inside the 128-column tile
+                auto chunk = [&](uint32_t (&raw)[32], int ch, auto mask_tag) {
+                    constexpr bool MASKED = decltype(mask_tag)::value;
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]);
+                    if (!PASS2) {
+                        if constexpr (MASKED) {
+                            const int lim = r + off - ch * 32;            // columns i <= lim are visible
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) if (i > lim) v[i] = -INFINITY;
+                        }
+                        float cm4[4] = {v[0], v[1], v[2], v[3]};      // four chains instead of one of 31
+#pragma unroll
+                        for (int i = 4; i < 32; ++i) cm4[i & 3] = fmaxf(cm4[i & 3], v[i]);
+                        const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
+                        const float mnew = fmaxf(mrun, cm * c);
+                        if (mnew != -INFINITY) {
+                            float2 part[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                            sum_exp2(v, c, mnew, part);
+                            Z = Z * fast_exp2(mrun - mnew) + ((part[0].x + part[0].y) + (part[1].x + part[1].y));
+                            mrun = mnew;
+                        }
+                    } else {
+                        const float4 *ls = reinterpret_cast<const float4 *>(lse_s + b * kTileRows + ch * 32);
+                        const int lim = r - off - ch * 32;                // columns i >= lim are visible
+                        const float2 c2 = make_float2(c, c);
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const float4 nl = ls[i4];                     // -lse of four query rows
+                            const float2 a01 = __ffma2_rn(make_float2(v[i4 * 4 + 0], v[i4 * 4 + 1]), c2, make_float2(nl.x, nl.y));
+                            const float2 a23 = __ffma2_rn(make_float2(v[i4 * 4 + 2], v[i4 * 4 + 3]), c2, make_float2(nl.z, nl.w));
+                            const float2 e01 = exp2_pair(a01, i4 * 2), e23 = exp2_pair(a23, i4 * 2 + 1);
+                            float p0 = e01.x, p1 = e01.y, p2 = e23.x, p3 = e23.y;
+                            if constexpr (MASKED) {
+                                if (i4 * 4 + 0 < lim) p0 = 0.f;
+                                if (i4 * 4 + 1 < lim) p1 = 0.f;
+                                if (i4 * 4 + 2 < lim) p2 = 0.f;
+                                if (i4 * 4 + 3 < lim) p3 = 0.f;
+                            }
+                            if constexpr (TAKE_MAX) {
+                                accA.x = fmaxf(accA.x, p0); accA.y = fmaxf(accA.y, p1);
+                                accB.x = fmaxf(accB.x, p2); accB.y = fmaxf(accB.y, p3);
+                            } else {
+                                accA = __fadd2_rn(accA, make_float2(p0, p1));
+                                accB = __fadd2_rn(accB, make_float2(p2, p3));
+                            }
+                        }
+                    }
+                };
+
+                // Only tiles the diagonal crosses pay for the mask: they run a separate instance.
+                auto tile_body = [&](auto mask_tag) {
+                    constexpr bool MASKED = decltype(mask_tag)::value;
+                    const uint32_t col0 = lane_addr + b * kTileRows;
+                    // A chunk the mask hides from all 32 rows of this warp is neither read nor
+                    // exponentiated (on a diagonal tile that is 6 of the 16 warp x chunk blocks).
+                    //   pass 1: column visible iff col <= row + off  -> hidden iff first col > last row + off
+                    //   pass 2: column visible iff col >= row - off  -> hidden iff last col < first row - off
+                    auto hidden = [&](int ch) {
+                        if (!MASKED) return false;
+                        return PASS2 ? (ch * 32 + 31 < q4 * 32 - off) : (ch * 32 > q4 * 32 + 31 + off);
+                    };
+                    const bool skip_a = hidden(half * 2), skip_b = hidden(half * 2 + 1);   // warp-uniform
+                    auto release = [&]() {
+                        tc_fence_before();               // all TMEM reads of this tile are done:
+                        __syncwarp();                    // hand the accumulator back before the last chunk's math
+                        if (lane == 0) mbar_arrive(bar_acc_empty(b));
+                    };
+                    if (!skip_a && !skip_b) {
+                        // this thread's 64 columns: the second 32 are in flight while the first are processed
+                        uint32_t ra[32], rb[32];
+                        tmem_ld32_async(col0, ra);
+                        tmem_ld_wait(ra);
+                        tmem_ld32_async(col0 + 32, rb);
+                        chunk(ra, half * 2, mask_tag);
+                        tmem_ld_wait(rb);
+                        release();
+                        chunk(rb, half * 2 + 1, mask_tag);
+                    } else if (skip_a && skip_b) {
+                        release();
+                    } else {
+                        const int which = skip_a ? 1 : 0;     // the one chunk some row of the warp can see
+                        uint32_t ra[32];
+                        tmem_ld32_async(col0 + 32 * which, ra);
+                        tmem_ld_wait(ra);
+                        release();
+                        chunk(ra, half * 2 + which, mask_tag);
+                    }
+                };
+                if (masked) tile_body(std::true_type{});
+                else tile_body(std::false_type{});
+            }
+            if (!alive) break;
+
+            // the two halves of a row meet: the second-half thread hands its result over
+            const uint32_t iph = it & 1u;
+            const float own = TAKE_MAX ? fmaxf(fmaxf(accA.x, accA.y), fmaxf(accB.x, accB.y))
+                                       : (accA.x + accA.y) + (accB.x + accB.y);
+            if (half == 1) {
+                if (!mbar_wait(bar_comb_empty, iph ^ 1u, abort_flag, status)) { alive = false; break; }
+                comb_s[r] = PASS2 ? make_float2(own, 0.f) : make_float2(mrun, Z);
+                mbar_arrive(bar_comb_full);
+            } else {
+                if (!mbar_wait(bar_comb_full, iph, abort_flag, status)) { alive = false; break; }
+                const float2 o = comb_s[r];
+                mbar_arrive(bar_comb_empty);
+                const int row = st * kTileRows + r;
+                if (!PASS2) {
+                    const float M = fmaxf(mrun, o.x);             // finite: column 0 of some tile is visible
+                    const float Zs = Z * fast_exp2(mrun - M) + o.y * fast_exp2(o.x - M);
+                    const float l2 = (row < geo.Tq) ? M + __log2f(Zs) : INFINITY;
+                    lse2[lse_row + row] = l2 - (fold.wa + fold.wb * (float)(row - (geo.Tq - 1)));   // +inf stays +inf
+                    if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
+                } else if (row < Tk) {
+                    float total = TAKE_MAX ? fmaxf(own, o.x) : own + o.x;
+                    if (fold.mean) total /= (float)(geo.Tq - (row > geo.P ? row - geo.P : 0));   // queries that see this key
+                    scores[(size_t)unit * Tk + row] = total;
+                }
+            }
+            ++it;
         }
     }
 
@@ -664,18 +702,22 @@ cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int unit
     e = cudaFuncSetAttribute(importance_kernel<D, STAGES, kPass2Max>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const long long resident = 2LL * sm_count();              // two persistent CTAs per SM
-    const long long super1 = (long long)units * ((geo.ntq + 1) / 2), super2 = (long long)units * ((geo.ntk + 1) / 2);
-    const unsigned grid1 = (unsigned)(super1 < resident ? super1 : resident);
-    const unsigned grid2 = (unsigned)(super2 < resident ? super2 : resident);
+    const long long items1 = (long long)units * geo.ntq, items2 = (long long)units * geo.ntk;
+    const unsigned grid1 = (unsigned)(items1 < resident ? items1 : resident);
+    const unsigned grid2 = (unsigned)(items2 < resident ? items2 : resident);
+    // units whose items are handed out longest-first at the end: about three items per CTA
+    auto tail_of = [&](int nt) { const long long v = (3 * resident + nt - 1) / nt; return (int)(v < units ? v : units); };
+    const int tail1 = tail_of(geo.ntq), tail2 = tail_of(geo.ntk);
+    // the passes' item counters: words 1 and 2 of the status block, zeroed with it at the start of the call
     if (first_pass)
-        importance_kernel<D, STAGES, kPass1><<<grid1, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)super1, c, lse2,
-                                                                              lse_out, scores, status);
+        importance_kernel<D, STAGES, kPass1><<<grid1, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)items1, tail1, c, lse2,
+                                                                              lse_out, scores, status, status + 1);
     if (take_max)
-        importance_kernel<D, STAGES, kPass2Max><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)super2, c, lse2,
-                                                                                 lse_out, scores, status);
+        importance_kernel<D, STAGES, kPass2Max><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)items2, tail2, c, lse2,
+                                                                                 lse_out, scores, status, status + 2);
     else
-        importance_kernel<D, STAGES, kPass2Sum><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)super2, c, lse2,
-                                                                                 lse_out, scores, status);
+        importance_kernel<D, STAGES, kPass2Sum><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)items2, tail2, c, lse2,
+                                                                                 lse_out, scores, status, status + 2);
     return cudaGetLastError();
 }
 
@@ -713,7 +755,7 @@ cudaError_t launch_importance(const void *Q, const void *K, float *scores, float
     geo.P = P;
     geo.ntq = (Tq + kTileRows - 1) / kTileRows;
     geo.ntk = (Tq + P + kTileRows - 1) / kTileRows;
-    if ((long long)units * geo.ntk > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    if ((long long)units * geo.ntk > 0x7FFF0000LL) return cudaErrorInvalidConfiguration;   // item numbers (plus the grid size) stay in an int
     Fold fold = {0.f, 0.f, statistic == EC_STAT_MEAN ? 1 : 0};
     if (statistic == EC_STAT_MOVING_AVERAGE) {
         const double lb = log2(beta);
