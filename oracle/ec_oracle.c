@@ -171,6 +171,51 @@ void eco_importance_prefix(const uint16_t *Q, const uint16_t *K, int U, int Tq, 
 }
 
 /*
+ * The forward pass whose attention Algorithm 1 takes as its input ("Input: ... attn"): the causal
+ * attention output of the prompt tokens, out[m] = sum_{n <= m+P} A[m][n] * v_n with A as in Eq. 1,
+ * together with each row's natural-log normaliser. Same geometry as eco_importance_prefix.
+ * Q: bf16 [U, Tq, D]; K, V: bf16 [U, P+Tq, D]; out: [U, Tq, D]; lse (nullable): [U, Tq].
+ */
+void eco_attention_prefix(const uint16_t *Q, const uint16_t *K, const uint16_t *V, int U, int Tq, int P, int D,
+                          double scale, double *out, double *lse)
+{
+    const int Tk = P + Tq;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < U; ++u) {
+        double *q = (double *)malloc(sizeof(double) * (size_t)Tq * D);
+        double *k = (double *)malloc(sizeof(double) * (size_t)Tk * D);
+        double *v = (double *)malloc(sizeof(double) * (size_t)Tk * D);
+        double *s = (double *)malloc(sizeof(double) * (size_t)Tk);
+        eco_widen_bf16(Q + (size_t)u * Tq * D, (int64_t)Tq * D, q);
+        eco_widen_bf16(K + (size_t)u * Tk * D, (int64_t)Tk * D, k);
+        eco_widen_bf16(V + (size_t)u * Tk * D, (int64_t)Tk * D, v);
+        for (int m = 0; m < Tq; ++m) {
+            const int last = m + P;
+            double mx = -INFINITY;
+            for (int n = 0; n <= last; ++n) {
+                double dot = 0.0;
+                for (int c = 0; c < D; ++c) dot += q[(size_t)m * D + c] * k[(size_t)n * D + c];
+                s[n] = scale * dot;
+                if (s[n] > mx) mx = s[n];
+            }
+            double Z = 0.0;
+            for (int n = 0; n <= last; ++n) Z += exp(s[n] - mx);
+            double *o = out + ((size_t)u * Tq + m) * D;
+            for (int c = 0; c < D; ++c) o[c] = 0.0;
+            for (int n = 0; n <= last; ++n) {
+                const double a = exp(s[n] - mx) / Z;
+                for (int c = 0; c < D; ++c) o[c] += a * v[(size_t)n * D + c];
+            }
+            if (lse) lse[(size_t)u * Tq + m] = mx + log(Z);
+        }
+        free(q);
+        free(k);
+        free(v);
+        free(s);
+    }
+}
+
+/*
  * Other statistics of the attention a key receives (Sec. 3.2 "Importance Metrics" lists summation,
  * moving average, maximum value and mean; the ablation on the importance metric compares moving
  * average, mean and sum). The paper prints no formulas for them; the readings taken here:

@@ -33,6 +33,8 @@ _lib.eco_importance_statistic.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_in
                                           C.c_double, _f64p]
 _lib.eco_importance_prefix.restype = None
 _lib.eco_importance_prefix.argtypes = [_u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _f64p, _f64p]
+_lib.eco_attention_prefix.restype = None
+_lib.eco_attention_prefix.argtypes = [_u16p, _u16p, _u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _f64p, _f64p]
 _lib.eco_layer_mean.restype = None
 _lib.eco_layer_mean.argtypes = [_f64p, C.c_int, C.c_int, C.c_int, _f64p]
 _lib.eco_group_mean.restype = None
@@ -98,6 +100,22 @@ def importance_prefix(Q: np.ndarray, K: np.ndarray, scale: float) -> Tuple[np.nd
     lse = np.empty(Q.shape[:-1], np.float64)
     _lib.eco_importance_prefix(_p(Q, _u16p), _p(K, _u16p), U, Tq, P, D, float(scale), _p(scores, _f64p), _p(lse, _f64p))
     return scores, lse
+
+
+def attention_prefix(Q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float) -> Tuple[np.ndarray, np.ndarray]:
+    """Causal attention output of the prompt tokens (the forward pass Algorithm 1 takes its attention
+    from). Q uint16 [..., Tq, D]; K, V uint16 [..., P+Tq, D]. Returns (out [..., Tq, D], lse [..., Tq])."""
+    Q, K, V = _bits(Q), _bits(K), _bits(V)
+    assert Q.shape[:-2] == K.shape[:-2] and Q.shape[-1] == K.shape[-1] and K.shape == V.shape
+    assert K.shape[-2] >= Q.shape[-2]
+    Tq, D = Q.shape[-2:]
+    P = K.shape[-2] - Tq
+    U = int(np.prod(Q.shape[:-2], dtype=np.int64))
+    out = np.empty(Q.shape, np.float64)
+    lse = np.empty(Q.shape[:-1], np.float64)
+    _lib.eco_attention_prefix(_p(Q, _u16p), _p(K, _u16p), _p(V, _u16p), U, Tq, P, D, float(scale),
+                              _p(out, _f64p), _p(lse, _f64p))
+    return out, lse
 
 
 STAT_SUM, STAT_MEAN, STAT_MAX, STAT_MOVING_AVERAGE = 0, 1, 2, 3

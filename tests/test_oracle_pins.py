@@ -471,3 +471,75 @@ def test_statistics_match_library_softmax(Tq, P, D):
                                A[:, -1, :].numpy(), rtol=1e-12)
     with pytest.raises(ValueError):
         orc.importance_statistic(qb, kb, 0.5, 7)
+
+
+# ------------------------------------------------------------------ attention output (the forward pass of Alg. 1's input)
+
+def test_attention_hand_example():
+    rows = _rows("attention_pow2.txt")
+    q = _bf16(np.array([[1.0, 0.0]] * 3).reshape(1, 3, 2))
+    k = _bf16(np.array([[0.0, 5.0], [1.0, 5.0], [2.0, 5.0]]).reshape(1, 3, 2))
+    v = _bf16(np.array([[1.0, 0.0], [0.0, 1.0], [4.0, -2.0]]).reshape(1, 3, 2))
+    out, lse = orc.attention_prefix(q, k, v, math.log(2.0))
+    want = np.array([[float(Fraction(int(a), int(b))), float(Fraction(int(c), int(d)))] for a, b, c, d, _ in rows])
+    np.testing.assert_allclose(out[0], want, rtol=1e-14, atol=1e-15)
+    np.testing.assert_allclose(lse[0], [math.log(float(r[4])) for r in rows], atol=1e-14)
+
+
+@pytest.mark.parametrize("Tq,P,D,scale", [(1, 0, 4, 1.0), (16, 0, 8, 0.5), (45, 0, 16, 0.25), (9, 13, 8, 0.4), (1, 20, 4, 1.0)])
+def test_attention_matches_library_softmax(Tq, P, D, scale):
+    rng = np.random.default_rng(Tq * 1000 + P * 10 + D)
+    qb = _rand_bits(rng, (2, Tq, D))
+    kb, vb = _rand_bits(rng, (2, P + Tq, D)), _rand_bits(rng, (2, P + Tq, D))
+    out, lse = orc.attention_prefix(qb, kb, vb, scale)
+    q = torch.from_numpy(orc.widen_bf16(qb))
+    k = torch.from_numpy(orc.widen_bf16(kb))
+    v = torch.from_numpy(orc.widen_bf16(vb))
+    logits = scale * q @ k.transpose(-1, -2)
+    m = torch.arange(Tq)[:, None]
+    n = torch.arange(P + Tq)[None, :]
+    logits = logits.masked_fill(n > m + P, float("-inf"))
+    np.testing.assert_allclose(out, (torch.softmax(logits, -1) @ v).numpy(), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(lse, torch.logsumexp(logits, -1).numpy(), rtol=1e-13, atol=1e-13)
+    # the normaliser is the one the importance function reports for the same inputs
+    _, lse_imp = orc.importance_prefix(qb, kb, scale)
+    np.testing.assert_array_equal(lse, lse_imp)
+
+
+def test_attention_zero_queries_is_running_mean_of_values():
+    # uniform attention: out[m] = mean of v_0 .. v_{m+P}
+    Tq, P, D = 23, 5, 8
+    rng = np.random.default_rng(3)
+    q = _bf16(np.zeros((1, Tq, D)))
+    kb, vb = _rand_bits(rng, (1, P + Tq, D)), _rand_bits(rng, (1, P + Tq, D))
+    out, lse = orc.attention_prefix(q, kb, vb, 0.9)
+    v = orc.widen_bf16(vb)[0]
+    want = np.cumsum(v, 0)[P:] / np.arange(P + 1, P + Tq + 1)[:, None]
+    np.testing.assert_allclose(out[0], want, rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(lse[0], np.log(np.arange(P + 1, P + Tq + 1)), atol=1e-13)
+
+
+def test_attention_invariants():
+    Tq, P, D = 31, 7, 8
+    rng = np.random.default_rng(11)
+    qb = _rand_bits(rng, (1, Tq, D), 2.0)
+    kb, vb = _rand_bits(rng, (1, P + Tq, D)), _rand_bits(rng, (1, P + Tq, D))
+    out, _ = orc.attention_prefix(qb, kb, vb, 0.5)
+    v = orc.widen_bf16(vb)[0]
+    # a convex combination of the visible value rows, coordinate by coordinate
+    for m in range(Tq):
+        vis = v[: m + P + 1]
+        assert np.all(out[0, m] <= vis.max(0) + 1e-12) and np.all(out[0, m] >= vis.min(0) - 1e-12)
+    # constant values come out unchanged whatever the attention is
+    const = _bf16(np.tile(np.array([1.5, -2.0, 0.25, 3.0, 0.0, 1.0, -1.0, 8.0], np.float32), (1, P + Tq, 1)))
+    out_c, _ = orc.attention_prefix(qb, kb, const, 0.5)
+    np.testing.assert_allclose(out_c[0], np.tile(orc.widen_bf16(const)[0, :1], (Tq, 1)), rtol=1e-13)
+    # summing the output rows weights every value row by the importance it received (Eq. 1's column sums)
+    scores, _ = orc.importance_prefix(qb, kb, 0.5)
+    np.testing.assert_allclose(out[0].sum(0), scores[0] @ v, rtol=1e-12, atol=1e-12)
+    # a change to a key or value the query cannot see changes nothing for that query
+    kb2, vb2 = kb.copy(), vb.copy()
+    kb2[0, P + 10:] = _rand_bits(rng, (Tq - 10, D))
+    vb2[0, P + 10:] = _rand_bits(rng, (Tq - 10, D))
+    out2, _ = orc.attention_prefix(qb, kb2, vb2, 0.5)
+    np.testing.assert_array_equal(out2[0, :10], out[0, :10])
