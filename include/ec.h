@@ -145,6 +145,27 @@ int ec_importance_from_lse(const void *Q_dev, const void *K_dev, const float *ls
                            void *ws_dev, size_t ws_bytes, void *stream);
 
 /*
+ * The forward pass itself, for callers that want the library to produce it: causal attention of
+ * the prompt tokens (Algorithm 1 "Input": the attention the method ranks tokens by is the one the
+ * model's forward pass computes), with each row's log-sum-exp, and, when `scores_dev` is given,
+ * the importance of Eq. 1 (Sec. 3.3) from that normaliser by the column-sum pass alone: three
+ * contractions for attention + importance instead of four.
+ *   out[m] = sum_{n <= m+P} softmax_n(scale*<q_m,k_n>) * v_n
+ *   Q_dev       bf16 [N, H, Tq, D]                                                  (in)
+ *   K_dev,V_dev bf16 [N, H, P+Tq, D]; P >= 0 earlier rows every query sees          (in)
+ *   out_dev     bf16 [N, H, Tq, D]: fp32 accumulation, probabilities rounded to bf16
+ *               before they meet V, one rounding of the normalised row at the end   (out)
+ *   lse_dev     fp32 [N, H, Tq] natural log-sum-exp of every query row, nullable    (out)
+ *   scores_dev  fp32 [N, H, P+Tq] importance as ec_importance_prefix gives it,
+ *               nullable (no column-sum pass then)                                  (out)
+ * Workspace, alignment, limits and status reporting as ec_importance_prefix
+ * (ec_importance_workspace(N, H, Tq, D) bytes). Deterministic.
+ */
+int ec_prefill_attention(const void *Q_dev, const void *K_dev, const void *V_dev, void *out_dev, float *lse_dev,
+                         float *scores_dev, int N, int H, int Tq, int P, int D, float scale,
+                         void *ws_dev, size_t ws_bytes, void *stream);
+
+/*
  * Synchronises `stream` and reports what the kernels recorded in the workspace's status
  * word: EC_OK, or EC_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are
  * then undefined but no out-of-bounds access happened). EC_ERR_CUDA on a runtime error.

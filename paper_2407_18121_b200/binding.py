@@ -24,7 +24,7 @@ EC_LAYER_SHARED = 1
 
 EXPORTS = (
     "ec_status_string", "ec_keep_count",
-    "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_statistic", "ec_importance_from_lse", "ec_device_status", "ec_selftest_wait_timeout",
+    "ec_importance_workspace", "ec_importance", "ec_importance_prefix", "ec_importance_statistic", "ec_importance_from_lse", "ec_prefill_attention", "ec_device_status", "ec_selftest_wait_timeout",
     "ec_select_merge_workspace", "ec_select_merge", "ec_select_compact_workspace", "ec_select_compact",
     "ec_cache_init", "ec_cache_init_ratio", "ec_cache_track_order", "ec_cache_concat", "ec_decode_workspace", "ec_decode_step", "ec_decode_steps",
     "ec_decode_noalloc_capacity", "ec_decode_step_noalloc", "ec_compress_host", "ec_decode_steps_host",
@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
     L.ec_importance_statistic.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, C.c_double, vp, sz, vp]
     L.ec_importance_from_lse.restype = i
     L.ec_importance_from_lse.argtypes = [vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
+    L.ec_prefill_attention.restype = i
+    L.ec_prefill_attention.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
     L.ec_device_status.restype = i
     L.ec_device_status.argtypes = [vp, vp]
     L.ec_selftest_wait_timeout.restype = i
@@ -190,6 +192,21 @@ def ec_importance_from_lse(Q: torch.Tensor, K: torch.Tensor, lse: torch.Tensor, 
     st = lib().ec_importance_from_lse(_ptr(Q), _ptr(K), _ptr(lse), _ptr(scores), N, H, T, D, float(scale),
                                       _ptr(ws), ws.numel() * ws.element_size(), _stream())
     _check(st, "ec_importance_from_lse")
+
+
+def ec_prefill_attention(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, out: torch.Tensor,
+                         lse: Optional[torch.Tensor], scores: Optional[torch.Tensor], scale: float,
+                         ws: torch.Tensor) -> None:
+    """Causal attention of the prompt tokens. Q: bf16 [N,H,Tq,D]; K, V: bf16 [N,H,P+Tq,D]; out (out): bf16
+    [N,H,Tq,D]; lse (out, optional): fp32 [N,H,Tq]; scores (out, optional): fp32 [N,H,P+Tq], the importance
+    from the column-sum pass alone; ws sized by ec_importance_workspace(N,H,Tq,D)."""
+    N, H, Tq, D = Q.shape
+    P = K.shape[2] - Tq
+    if K.shape != V.shape or tuple(out.shape) != tuple(Q.shape):
+        raise ValueError("K and V must have one shape, out the shape of Q")
+    st = lib().ec_prefill_attention(_ptr(Q), _ptr(K), _ptr(V), _ptr(out), _ptr(lse), _ptr(scores), N, H, Tq, P, D,
+                                    float(scale), _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(st, "ec_prefill_attention")
 
 
 def ec_device_status(ws: torch.Tensor) -> int:

@@ -173,6 +173,27 @@ int ec_importance_from_lse(const void *Q, const void *K, const float *lse, float
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 
+int ec_prefill_attention(const void *Q, const void *K, const void *V, void *out, float *lse, float *scores, int N, int H,
+                         int Tq, int P, int D, float scale, void *ws, size_t ws_bytes, void *stream)
+{
+    ec::NvtxRange nvtx_range("ec_prefill_attention");
+    if (!Q || !K || !V || !out) return EC_ERR_NULL;
+    if (P < 0 || Tq < 1 || (long long)P + Tq > kMaxT) return EC_ERR_SHAPE;
+    int st = check_shape(N, H, Tq + P, D);
+    if (st != EC_OK) return st;
+    if (!(scale > 0.f) || !isfinite(scale)) return EC_ERR_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(out, 16) || (lse && !aligned(lse, 16)) ||
+        (scores && !aligned(scores, 16)))
+        return EC_ERR_ALIGN;
+    if (!ws || ws_bytes < ec::importance_workspace_bytes(N, H, Tq, D)) return EC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EC_ERR_ALIGN;
+    cudaError_t e = ec::launch_attention(Q, K, V, out, lse, N, H, Tq, P, D, scale, ws, (cudaStream_t)stream);
+    if (e == cudaSuccess && scores)
+        e = ec::launch_importance(Q, K, scores, nullptr, ec::kLseInWorkspace, N, H, Tq, P, D, scale, EC_STAT_SUM, 0.0, ws,
+                                  (cudaStream_t)stream);
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
 int ec_selftest_wait_timeout(void *ws, unsigned limit_us, void *stream)
 {
     if (!ws) return EC_ERR_NULL;

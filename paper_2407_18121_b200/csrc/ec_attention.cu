@@ -1,0 +1,467 @@
+// Causal attention of the prompt tokens that also hands out each row's softmax normaliser
+// (the forward pass Algorithm 1 takes its attention from, Alg. 1 "Input"): with the normaliser
+// known, the importance of Eq. 1 costs one more contraction (the column-sum pass) instead of two.
+//   out[m] = sum_{n <= m+P} softmax_n(scale*<q_m,k_n>) * v_n        lse[m] = log sum_{n <= m+P} exp(scale*<q_m,k_n>)
+// One work item is a 128-row query tile of one unit. Its key tiles stream from the diagonal down
+// to tile 0; for each, S = Q K^T goes into TMEM (tcgen05.mma, both operands K-major from TMA-staged
+// shared memory), the softmax warps turn S into P = 2^(c*S - m) in bf16, written to shared memory in
+// the same swizzled K-major layout, and a second tcgen05.mma accumulates O += P V in TMEM with the V
+// tile as an MN-major operand (rows of V are contiguous along the head dimension). The running
+// maximum m is only raised when a tile exceeds it by more than 8 (in the log2 domain), so the
+// accumulator in TMEM is rescaled rarely: P never exceeds 2^8 and the result does not depend on when
+// m is raised. Two threads share a query row (64 columns of S each); the row maximum of a tile is
+// exchanged through shared memory, so both use the same m and the same P scaling.
+// Roles: warp 0 TMA, warp 1 MMA issue + TMEM allocation, warps 2..9 softmax. One CTA per SM (the
+// tiles of Q, two stages of K and V and P take 192 KB at head dimension 128). Items are handed out
+// as in the importance kernels (a counter, longest first inside a unit and over the last units).
+// Every mbarrier wait is bounded in time; on expiry the CTA records a status word and leaves.
+#include "ec_tc.cuh"
+
+#include <type_traits>
+
+namespace ec {
+
+namespace {
+
+constexpr int kAttnThreads = 320;
+constexpr int kAttnSched = 4;
+constexpr int kAttnTmemCols = 512;        // S: 2 x 128 columns, O: up to 128 columns
+constexpr float kRaiseBy = 8.f;           // the running maximum moves only when a tile exceeds it by this much
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// MN-major operand with the 128-byte swizzle: 64 contiguous elements of the MN dimension per
+// 128-byte row, 8 rows (steps of the contraction index) per 1024-byte group; `lbo` bytes to the next
+// 64 elements of the MN dimension, `sbo` bytes to the next 8 steps of the contraction index.
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+template <int D>
+struct AttnSmem {
+    static constexpr int kTile = kTileRows * D * 2;                       // a Q, K or V tile
+    static constexpr int kPBytes = kTileRows * kTileRows * 2;             // P: 128 x 128 bf16
+    static constexpr int kQ = 0;
+    static constexpr int kK0 = kTile;
+    static constexpr int kV0 = kK0 + 2 * kTile;
+    static constexpr int kP = kV0 + 2 * kTile;
+    static constexpr int kExch = kP + kPBytes;                            // [2 S buffers][2 halves][128] row maxima
+    static constexpr int kLsum = kExch + 2 * 2 * kTileRows * 4;           // [2 halves][128] row sums
+    static constexpr int kBars = kLsum + 2 * kTileRows * 4;
+    // q_full, q_empty, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], x_rdv[2],
+    // p_full, pv_done, o_free, l_rdv, sched_full[4], sched_empty[4]
+    static constexpr int kNumBars = 2 + 4 + 4 + 4 + 2 + 4 + 2 * kAttnSched;
+    static constexpr int kTmemSlot = kBars + kNumBars * 8;
+    static constexpr int kAbort = kTmemSlot + 4;
+    static constexpr int kSchedItems = (kAbort + 4 + 15) & ~15;
+    static constexpr int kTotal = kSchedItems + kAttnSched * 16;
+    static constexpr int kDynBytes = kTotal + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, const Geometry geo, int n_items, int tail_units, float c,
+                 __nv_bfloat16 *__restrict__ out, float *__restrict__ lse2, float *__restrict__ lse_out,
+                 int *__restrict__ status, int *__restrict__ next_item)
+{
+    using L = AttnSmem<D>;
+    constexpr int kTile = L::kTile;
+    constexpr int kBoxes = D / 64;
+    constexpr int kBoxBytes = kTileRows * 128;
+    // S = Q K^T: M = 128 queries, N = 128 keys, both K-major
+    constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kTileRows >> 3) << 17) | ((kTileRows >> 4) << 24);
+    // O += P V: M = 128 queries, N = D, A (P) K-major, B (V) MN-major
+    constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((D >> 3) << 17) | ((kTileRows >> 4) << 24);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + L::kBars;
+    const uint32_t bar_q_full = bars, bar_q_empty = bars + 8u;
+    auto bar_k_full = [&](uint32_t s) { return bars + 8u * (2 + s); };
+    auto bar_k_empty = [&](uint32_t s) { return bars + 8u * (4 + s); };
+    auto bar_v_full = [&](uint32_t s) { return bars + 8u * (6 + s); };
+    auto bar_v_empty = [&](uint32_t s) { return bars + 8u * (8 + s); };
+    auto bar_s_full = [&](uint32_t b) { return bars + 8u * (10 + b); };
+    auto bar_s_empty = [&](uint32_t b) { return bars + 8u * (12 + b); };
+    auto bar_x_rdv = [&](uint32_t b) { return bars + 8u * (14 + b); };
+    const uint32_t bar_p_full = bars + 8u * 16, bar_pv_done = bars + 8u * 17, bar_o_free = bars + 8u * 18,
+                   bar_l_rdv = bars + 8u * 19;
+    auto bar_sched_full = [&](uint32_t k) { return bars + 8u * (20 + k); };
+    auto bar_sched_empty = [&](uint32_t k) { return bars + 8u * (20 + kAttnSched + k); };
+    float *exch_s = reinterpret_cast<float *>(base_ptr + L::kExch);
+    float *lsum_s = reinterpret_cast<float *>(base_ptr + L::kLsum);
+    int4 *sched_s = reinterpret_cast<int4 *>(base_ptr + L::kSchedItems);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + L::kTmemSlot);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + L::kAbort);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nts = geo.ntq;
+    const int grid_n = (int)gridDim.x;
+
+    if (threadIdx.x == 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    }
+    if (threadIdx.x == 0) *abort_flag = *reinterpret_cast<volatile int *>(status);
+    __syncthreads();
+    if (*abort_flag) return;
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar_q_full, 1);
+        mbar_init(bar_q_empty, 1);
+        for (uint32_t s = 0; s < 2; ++s) {
+            mbar_init(bar_k_full(s), 1); mbar_init(bar_k_empty(s), 1);
+            mbar_init(bar_v_full(s), 1); mbar_init(bar_v_empty(s), 1);
+            mbar_init(bar_s_full(s), 1); mbar_init(bar_s_empty(s), 8);
+            mbar_init(bar_x_rdv(s), 8 * 32);
+        }
+        mbar_init(bar_p_full, 8 * 32);
+        mbar_init(bar_pv_done, 1);
+        mbar_init(bar_o_free, 8);
+        mbar_init(bar_l_rdv, 8 * 32);
+        for (uint32_t k = 0; k < (uint32_t)kAttnSched; ++k) {
+            mbar_init(bar_sched_full(k), 1);
+            mbar_init(bar_sched_empty(k), 1 + 8);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + (uint32_t)L::kTmemSlot), "r"((uint32_t)kAttnTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base + 2u * kTileRows;            // O after the two S buffers
+
+    // `it` counts items, `tg` counts key tiles; slots and barrier phases derive from them in every role.
+    uint32_t it = 0, tg = 0;
+    bool alive = true;
+
+    // item -> unit, query tile, first (highest) key tile, number of key tiles; the order is the one
+    // the importance kernels use (see there): longest first inside a unit and over the last units.
+    const int n_units = n_items / nts, head_items = (n_units - tail_units) * nts;
+    auto decode_item = [&](int item, int &unit, int &st, int &first, int &count) {
+        int k;
+        if (item < head_items) {
+            unit = item / nts;
+            k = item - unit * nts;
+        } else {
+            const int j = item - head_items;
+            k = j / tail_units;
+            unit = (n_units - tail_units) + (j - k * tail_units);
+        }
+        st = nts - 1 - k;
+        first = geo.jmax(st);
+        count = first + 1;
+    };
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            uint32_t k_armed = 0, v_armed = 0, q_armed = 0;
+            int item = (int)blockIdx.x;
+            for (uint32_t k = 0; alive; ++k) {
+                const uint32_t sl = k % kAttnSched, sph = (k / kAttnSched) & 1u;
+                if (!mbar_wait(bar_sched_empty(sl), sph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                int unit = -1, st = 0, first = 0, count = 0;
+                if (item < n_items) decode_item(item, unit, st, first, count);
+                sched_s[sl] = make_int4(unit, st, first, count);
+                mbar_arrive(bar_sched_full(sl));
+                if (unit < 0) break;
+                const int next = grid_n + atomicAdd(next_item, 1);
+                for (int t = 0; t < count; ++t, ++tg) {
+                    const uint32_t s = tg & 1u, ph = (tg >> 1) & 1u;
+                    const int row0 = (first - t) * kTileRows;
+                    if (!mbar_wait(bar_k_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    mbar_expect_tx(bar_k_full(s), kTile);
+#pragma unroll
+                    for (int bx = 0; bx < kBoxes; ++bx)
+                        tma_load_3d(base + L::kK0 + s * kTile + bx * kBoxBytes, &map_k, bx * 64, row0, unit, bar_k_full(s));
+                    k_armed = tg + 1;
+                    if (t == 0) {
+                        if (!mbar_wait(bar_q_empty, (it + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                        mbar_expect_tx(bar_q_full, kTile);
+#pragma unroll
+                        for (int bx = 0; bx < kBoxes; ++bx)
+                            tma_load_3d(base + L::kQ + bx * kBoxBytes, &map_q, bx * 64, st * kTileRows, unit, bar_q_full);
+                        q_armed = it + 1;
+                    }
+                    if (!mbar_wait(bar_v_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    mbar_expect_tx(bar_v_full(s), kTile);
+#pragma unroll
+                    for (int bx = 0; bx < kBoxes; ++bx)
+                        tma_load_3d(base + L::kV0 + s * kTile + bx * kBoxBytes, &map_v, bx * 64, row0, unit, bar_v_full(s));
+                    v_armed = tg + 1;
+                }
+                ++it;
+                item = next;
+            }
+            if (*abort_flag) {
+                // let copies that are still in flight land before the CTA gives its memory back
+                if (q_armed > 0) mbar_wait(bar_q_full, (q_armed - 1u) & 1u, abort_flag, status, 200000ull);
+                for (uint32_t t = k_armed > 2u ? k_armed - 2u : 0; t < k_armed; ++t)
+                    mbar_wait(bar_k_full(t & 1u), (t >> 1) & 1u, abort_flag, status, 200000ull);
+                for (uint32_t t = v_armed > 2u ? v_armed - 2u : 0; t < v_armed; ++t)
+                    mbar_wait(bar_v_full(t & 1u), (t >> 1) & 1u, abort_flag, status, 200000ull);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            // S(tile x) = Q K_x^T into S buffer x & 1
+            auto issue_s = [&](uint32_t x) -> bool {
+                const uint32_t s = x & 1u, ph = (x >> 1) & 1u;
+                if (!mbar_wait(bar_s_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) return false;
+                if (!mbar_wait(bar_k_full(s), ph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) return false;
+                tc_fence_after();
+                const uint32_t a0 = base + L::kQ, b0 = base + L::kK0 + s * kTile;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (uint32_t)(kk / 4) * kBoxBytes + (uint32_t)(kk % 4) * 32u;
+                    umma_bf16(tmem_base + s * kTileRows, umma_desc(a0 + off), umma_desc(b0 + off), kIdescS, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(bar_k_empty(s));
+                umma_commit(bar_s_full(s));
+                return true;
+            };
+            for (uint32_t k = 0; alive; ++k) {
+                const uint32_t sl = k % kAttnSched, sph = (k / kAttnSched) & 1u;
+                if (!mbar_wait(bar_sched_full(sl), sph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                const int4 d = sched_s[sl];
+                mbar_arrive(bar_sched_empty(sl));
+                if (d.x < 0) break;
+                const int count = d.w;
+                if (!mbar_wait(bar_q_full, it & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                if (!issue_s(tg)) { alive = false; break; }
+                for (int t = 0; t < count; ++t, ++tg) {
+                    // the next tile's S is issued first, so that the tensor cores work under this tile's softmax
+                    if (t + 1 < count) { if (!issue_s(tg + 1u)) { alive = false; break; } }
+                    else umma_commit(bar_q_empty);                    // the item's last S is on its way: Q is free after it
+                    const uint32_t s = tg & 1u, ph = (tg >> 1) & 1u;
+                    if (!mbar_wait(bar_p_full, tg & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    if (!mbar_wait(bar_v_full(s), ph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    // the previous item's output has been read out of TMEM before this item overwrites it
+                    if (t == 0 && !mbar_wait(bar_o_free, (it + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t p0 = base + L::kP, v0 = base + L::kV0 + s * kTile;
+#pragma unroll
+                    for (int kk = 0; kk < kTileRows / 16; ++kk) {     // 16 keys per instruction
+                        const uint32_t aoff = (uint32_t)(kk / 4) * kBoxBytes + (uint32_t)(kk % 4) * 32u;
+                        umma_bf16(tmem_o, umma_desc(p0 + aoff), umma_desc_mn(v0 + (uint32_t)kk * 2048u, kBoxBytes, 1024u),
+                                  kIdescO, (t > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(bar_v_empty(s));
+                    umma_commit(bar_pv_done);
+                }
+                ++it;
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- softmax warps
+        const int q4 = warp & 3;                              // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                     // which 64 columns of S, which half of O's columns
+        const int r = q4 * 32 + lane;                         // row of the query tile = TMEM lane
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const uint32_t o_addr = tmem_o + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(half * (D / 2));
+        // this thread's 128 bytes of a row of P: box `half`, row r, eight 16-byte chunks XOR-swizzled by the row
+        uint8_t *p_row = base_ptr + L::kP + half * kBoxBytes + r * 128;
+        const float2 c2 = make_float2(c, c);
+        for (uint32_t k = 0; alive; ++k) {
+            const uint32_t sl = k % kAttnSched, sph = (k / kAttnSched) & 1u;
+            if (!mbar_wait(bar_sched_full(sl), sph, abort_flag, status)) { alive = false; break; }
+            const int4 d = sched_s[sl];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_sched_empty(sl));
+            if (d.x < 0) break;
+            const int unit = d.x, st = d.y, first = d.z, count = d.w;
+            float m_ref = -INFINITY, l = 0.f;                 // running maximum (log2 domain) and this half's row sum
+            for (int t = 0; t < count; ++t, ++tg) {
+                const uint32_t b = tg & 1u, bph = (tg >> 1) & 1u;
+                const int tile = first - t;
+                const int off = (st - tile) * kTileRows + geo.P;          // column col of the tile is visible iff col <= r + off
+                if (!mbar_wait(bar_s_full(b), bph, abort_flag, status)) { alive = false; break; }
+                tc_fence_after();
+                uint32_t ra[32], rb[32];
+                tmem_ld32_async(lane_base + b * kTileRows + half * 64, ra);
+                tmem_ld32_async(lane_base + b * kTileRows + half * 64 + 32, rb);
+                tmem_ld_wait(ra);
+                tmem_ld_wait(rb);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_s_empty(b));
+                float v[64];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) { v[i] = __uint_as_float(ra[i]); v[32 + i] = __uint_as_float(rb[i]); }
+                if (off < kTileRows - 1) {
+                    const int lim = r + off - half * 64;
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) if (i > lim) v[i] = -INFINITY;
+                }
+                float mx4[4] = {v[0], v[1], v[2], v[3]};
+#pragma unroll
+                for (int i = 4; i < 64; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], v[i]);
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                // both halves of the row agree on the tile's maximum before either scales anything
+                exch_s[(b * 2 + half) * kTileRows + r] = mx;
+                mbar_arrive(bar_x_rdv(b));
+                if (!mbar_wait(bar_x_rdv(b), bph, abort_flag, status)) { alive = false; break; }
+                const float tile_max = fmaxf(mx, exch_s[(b * 2 + (half ^ 1)) * kTileRows + r]) * c;
+                float factor = 1.f;
+                bool rescale = false;
+                if (tile_max > m_ref + kRaiseBy) {            // also the first tile that shows this row anything
+                    if (m_ref != -INFINITY) { rescale = true; factor = fast_exp2(m_ref - tile_max); }
+                    m_ref = tile_max;
+                }
+                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                const float2 nm = make_float2(-m_use, -m_use);
+                float2 sum2 = make_float2(0.f, 0.f);
+                uint32_t pk[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float2 a = __ffma2_rn(make_float2(v[2 * i], v[2 * i + 1]), c2, nm);
+                    const float2 e = exp2_pair(a, i);
+                    sum2 = __fadd2_rn(sum2, e);
+                    pk[i] = pack2(e.x, e.y);
+                }
+                l = l * factor + (sum2.x + sum2.y);
+                // P's buffer is free, and O is at rest, once the previous tile's P V has completed
+                if (t > 0) {
+                    if (!mbar_wait(bar_pv_done, (tg - 1u) & 1u, abort_flag, status)) { alive = false; break; }
+                    tc_fence_after();
+                }
+                // TMEM loads and stores are warp-wide instructions: if any row of the warp raises its
+                // maximum, the whole warp runs them (the other rows multiply by one, which changes nothing)
+                if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+                    for (int j = 0; j < D / 64; ++j) {
+                        uint32_t ro[32];
+                        tmem_ld32_async(o_addr + 32 * j, ro);
+                        tmem_ld_wait(ro);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) ro[i] = __float_as_uint(__uint_as_float(ro[i]) * factor);
+                        tmem_st32(o_addr + 32 * j, ro);
+                    }
+                    tmem_st_wait();
+                }
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc)
+                    *reinterpret_cast<uint4 *>(p_row + ((cc ^ (r & 7)) << 4)) =
+                        make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor cores
+                tc_fence_before();
+                mbar_arrive(bar_p_full);
+            }
+            if (!alive) break;
+
+            // the item's last P V has completed: normalise and store the rows, report the normaliser
+            if (!mbar_wait(bar_pv_done, (tg - 1u) & 1u, abort_flag, status)) { alive = false; break; }
+            tc_fence_after();
+            lsum_s[half * kTileRows + r] = l;
+            mbar_arrive(bar_l_rdv);
+            if (!mbar_wait(bar_l_rdv, it & 1u, abort_flag, status)) { alive = false; break; }
+            const float l_tot = l + lsum_s[(half ^ 1) * kTileRows + r];
+            const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+            const int row = st * kTileRows + r;
+#pragma unroll
+            for (int j = 0; j < D / 64; ++j) {
+                uint32_t ro[32];
+                tmem_ld32_async(o_addr + 32 * j, ro);
+                tmem_ld_wait(ro);
+                if (row < geo.Tq) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(out + ((size_t)unit * geo.Tq + row) * D + half * (D / 2) + 32 * j);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float f[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(ro[8 * q + i]) * inv;
+                        dst[q] = pack8(f);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_o_free);
+            if (half == 0) {
+                const float l2 = (row < geo.Tq) ? m_ref + __log2f(l_tot) : INFINITY;
+                lse2[(size_t)unit * geo.ntq * kTileRows + row] = l2;                 // padded layout of the column-sum pass
+                if (lse_out && row < geo.Tq) lse_out[(size_t)unit * geo.Tq + row] = l2 * kLn2;
+            }
+            ++it;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kAttnTmemCols) : "memory");
+    }
+}
+
+template <int D>
+cudaError_t launch_attention_t(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, int units,
+                               const Geometry &geo, float c, void *out, float *lse2, float *lse_out, int *status,
+                               cudaStream_t stream)
+{
+    constexpr int smem = AttnSmem<D>::kDynBytes;
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    const long long resident = sm_count();                        // one persistent CTA per SM
+    const long long items = (long long)units * geo.ntq;
+    const unsigned grid = (unsigned)(items < resident ? items : resident);
+    const long long tail = (3 * resident + geo.ntq - 1) / geo.ntq;
+    attention_kernel<D><<<grid, kAttnThreads, smem, stream>>>(mq, mk, mv, geo, (int)items, (int)(tail < units ? tail : units), c,
+                                                              static_cast<__nv_bfloat16 *>(out), lse2, lse_out, status,
+                                                              status + 3);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// Q: [units, Tq, D]; K, V: [units, P + Tq, D]; out: [units, Tq, D] bf16; lse_out (nullable): [units, Tq].
+// Leaves the padded log2-domain normaliser in the workspace (behind the status block), where the
+// column-sum pass of the importance kernels reads it. Zeroes the status block first.
+cudaError_t launch_attention(const void *Q, const void *K, const void *V, void *out, float *lse_out, int N, int H,
+                             int Tq, int P, int D, float scale, void *ws, cudaStream_t stream)
+{
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, stream);
+    if (e != cudaSuccess) return e;
+    int *status = static_cast<int *>(ws);
+    float *lse2 = reinterpret_cast<float *>(static_cast<char *>(ws) + kStatusBytes);
+    const int units = N * H;
+    Geometry geo;
+    geo.Tq = Tq;
+    geo.P = P;
+    geo.ntq = (Tq + kTileRows - 1) / kTileRows;
+    geo.ntk = (Tq + P + kTileRows - 1) / kTileRows;
+    if ((long long)units * geo.ntk > 0x7FFF0000LL) return cudaErrorInvalidConfiguration;
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, Q, units, Tq, D) || !make_map(&mk, K, units, Tq + P, D) || !make_map(&mv, V, units, Tq + P, D))
+        return cudaErrorInvalidValue;
+    const float c = scale * kLog2e;
+    if (D == 128) return launch_attention_t<128>(mq, mk, mv, units, geo, c, out, lse2, lse_out, status, stream);
+    return launch_attention_t<64>(mq, mk, mv, units, geo, c, out, lse2, lse_out, status, stream);
+}
+
+}  // namespace ec

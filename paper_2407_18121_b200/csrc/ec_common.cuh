@@ -79,6 +79,10 @@ cudaError_t launch_importance(const void *Q, const void *K, float *scores, float
                               int N, int H, int Tq, int P, int D, float scale, int statistic, double beta, void *ws,
                               cudaStream_t stream);
 size_t importance_workspace_bytes(int N, int H, int T, int D);
+// passed as launch_importance's lse_in: the normaliser already lies in the workspace (see there)
+static const float *const kLseInWorkspace = reinterpret_cast<const float *>(static_cast<uintptr_t>(1));
+cudaError_t launch_attention(const void *Q, const void *K, const void *V, void *out, float *lse_out, int N, int H,
+                             int Tq, int P, int D, float scale, void *ws, cudaStream_t stream);
 cudaError_t launch_wait_selftest(void *ws, unsigned limit_us, cudaStream_t stream);
 
 cudaError_t launch_select(const float *scores, int units, int T, int n_keep, int share, int protect_ends,
