@@ -50,7 +50,7 @@ OTHER_WORKLOADS = ("llava7b_b1", "llava13b_b4", "long8k")
 # launch by the number of units (every unit streams its own rows once: traffic is proportional to
 # units); valid only for the kernel source it was taken on (sha1 prefix of csrc/ec_decode.cu),
 # otherwise reported as null.
-DECODE_TRAFFIC = {"source_sha1": "", "llava7b_b8": None}
+DECODE_TRAFFIC = {"source_sha1": "2c38c94c6bc1", "llava7b_b8": 4 * (270075904 + 3239168)}
 
 
 def decode_traffic(workload: str):
@@ -515,6 +515,41 @@ def run_ours(args, w: wl.Workload):
         graph_ms = g0.elapsed_time(g1) / reps
         del g
 
+    # The fused form of the prompt stage (attention output + importance in one call: three contractions
+    # instead of the two of ec_importance plus the two of an attention kernel), timed on the same
+    # tensors beside the pass; it is not part of the timed pass, whose importance call is ec_importance.
+    attn = None
+    if not args.no_attention:
+        attn_out = torch.empty_like(dp.Q)
+        attn_scores = torch.empty_like(dp.sess.scores)
+
+        def attn_call(with_scores):
+            ec.ec_prefill_attention(dp.Q, dp.K, dp.V, attn_out, None, attn_scores if with_scores else None, wr.scale,
+                                    dp.sess.ws_imp)
+
+        attn_ms = {}
+        for with_scores in (False, True):
+            for _ in range(3):
+                attn_call(with_scores)
+            barrier()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(3, min(args.steps, 10))
+            a0.record(stream)
+            for _ in range(reps):
+                attn_call(with_scores)
+            a1.record(stream)
+            barrier()
+            attn_ms[with_scores] = a0.elapsed_time(a1) / reps
+        if ec.ec_device_status(dp.sess.ws_imp) != ec.EC_OK:
+            raise SystemExit("device status after ec_prefill_attention")
+        one = 1.0 * D * T * (T + 1) * N * H                        # flops of one causal contraction
+        attn = {"attention_ms": attn_ms[False], "attention_tflops": 2 * one / (attn_ms[False] * 1e-3) / 1e12,
+                "attention_and_importance_ms": attn_ms[True],
+                "attention_and_importance_tflops": 3 * one / (attn_ms[True] * 1e-3) / 1e12,
+                "note": ("ec_prefill_attention without / with the column-sum pass; flops = 2*D per visible "
+                         "(query, key) pair and contraction: two contractions for the attention, three with the importance")}
+        del attn_out, attn_scores
+
     # end to end: inputs start in pinned host memory, results are read back every pass. Two passes are
     # in flight, each with its own session, stream and host result buffers, so that the upload of the
     # next pass's prompt overlaps the decode loop of this one (a serving loop with double buffering);
@@ -593,6 +628,7 @@ def run_ours(args, w: wl.Workload):
         "roofline": roofline,
         "merge": dict(mrg, note="whole ec_select_merge call (selection + merge kernels)"),
         "importance": imp,
+        "prefill_attention": attn,
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "pipeline": "two passes in flight: the next pass's prompt upload overlaps this pass's decode loop"},
@@ -631,6 +667,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     ap.add_argument("--no-per-workload", action="store_true", help="skip the other configurations")
+    ap.add_argument("--no-attention", action="store_true", help="skip the timing of ec_prefill_attention")
     ap.add_argument("--no-read-peak", action="store_true", help="skip the read-only stream measurement")
     ap.add_argument("--per-workload-passes", type=int, default=4)
     args = ap.parse_args()

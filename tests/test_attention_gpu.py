@@ -9,7 +9,7 @@ import torch
 from oracle import ec_oracle as orc
 from paper_2407_18121_b200 import binding as ec
 from paper_2407_18121_b200 import workloads as wl
-from tests.helpers import (SCORE_RTOL, Guarded, assert_bf16_close, assert_rel_close, dev_bf16, host_bits, host_f64,
+from helpers import (SCORE_RTOL, Guarded, assert_bf16_close, assert_rel_close, dev_bf16, host_bits, host_f64,
                            scratch)
 
 pytestmark = pytest.mark.gpu
@@ -112,3 +112,38 @@ def test_prefill_attention_refuses_bad_arguments():
     with pytest.raises(ec.EcError) as e:
         ec.ec_prefill_attention(Q, Q, Q, out, None, None, 1.0, ws[:128])
     assert e.value.status == ec.EC_ERR_WORKSPACE
+
+
+def _check_sampled_rows(w, problems, units, row_blocks):
+    """The whole batch of `problems` on the GPU in one call; the oracle on sampled row blocks of sampled units
+    (a block of query rows m0..m1 of a unit is the prefix form with P = m0 earlier keys: the same rows)."""
+    Qb, Kb, Vb = wl.prompt(w, problems)
+    N, H, T, D = Qb.shape
+    out, lse, scores = run_attention(Qb, Kb, Vb, w.scale)
+    out_h, lse_h, scores_h = host_f64(out), host_f64(lse), host_f64(scores)
+    assert np.isfinite(out_h).all()
+    np.testing.assert_allclose(scores_h.sum(-1), T, rtol=1e-3)
+    for (n, h) in units:
+        for (m0, m1) in row_blocks:
+            want_out, want_lse = orc.attention_prefix(Qb[n, h, m0:m1][None], Kb[n, h, :m1][None], Vb[n, h, :m1][None], w.scale)
+            err = np.abs(out_h[n, h, m0:m1] - want_out[0])
+            assert (err <= 2e-2 + 2.0 ** -8 * np.abs(want_out[0])).all(), (n, h, m0, float(err.max()))
+            np.testing.assert_allclose(lse_h[n, h, m0:m1], want_lse[0], rtol=1e-3, atol=1e-3)
+    # the scores are the ones the two-pass call gives (same kernels for the column sums, another normaliser)
+    Q, K = dev_bf16(Qb), dev_bf16(Kb)
+    ref = torch.empty_like(scores)
+    ws = scratch(ec.ec_importance_workspace(N, H, T, D))
+    ec.ec_importance(Q, K, ref, None, w.scale, ws)
+    torch.testing.assert_close(scores, ref, rtol=2e-4, atol=0)
+
+
+def test_prefill_attention_7b_batch8_shapes_full_length():
+    # 1024-token prompts of the batch-8 7B configuration, 8 problems = 256 units in one launch
+    w = wl.WORKLOADS["llava7b_b8"]
+    _check_sampled_rows(w, list(range(8)), [(0, 0), (3, 17), (7, 31)], [(0, 130), (500, 640), (896, 1024)])
+
+
+def test_prefill_attention_long_context_units_full_length():
+    # 8192-token units of the long-context configuration (64 key tiles per query tile at the end)
+    w = wl.WORKLOADS["long8k"]
+    _check_sampled_rows(w, [0, 1], [(0, 0), (1, 31)], [(0, 129), (4000, 4100), (8064, 8192)])
