@@ -576,6 +576,24 @@ def test_importance_statistics_match_oracle(N, H, Tq, P, D, stat, beta):
     assert_rel_close(lse.t, want_lse, 1e-3, atol=1e-3, what="lse is the plain one whatever the statistic")
 
 
+@pytest.mark.parametrize("beta", [0.5, 0.1])
+def test_moving_average_long_prompt_small_factor(beta):
+    # the exponent of a query's weight reaches -Tq*log2(1/beta) (tens of thousands for the oldest queries); it is
+    # counted from the last query, so the newest queries, which carry the weight, keep an exact exponent
+    N, H, Tq, D = 1, 2, 4096, 128
+    rng = np.random.default_rng(int(beta * 100))
+    Qb, Kb = rand_bits(rng, (N, H, Tq, D)), rand_bits(rng, (N, H, Tq, D))
+    scale = 1.0 / math.sqrt(D)
+    want = orc.importance_statistic(Qb, Kb, scale, orc.STAT_MOVING_AVERAGE, beta)
+    scores = Guarded((N, H, Tq), torch.float32, fill=float("nan"))
+    ws = scratch(ec.ec_importance_workspace(N, H, Tq, D))
+    ec.ec_importance_statistic(dev_bf16(Qb), dev_bf16(Kb), scores.t, None, scale, ec.EC_STAT_MOVING_AVERAGE, beta, ws)
+    assert ec.ec_device_status(ws) == ec.EC_OK
+    scores.check("scores")
+    assert_rel_close(scores.t, want, SCORE_RTOL, atol=1e-30, what=f"moving average, beta {beta}")
+    np.testing.assert_allclose(host_f64(scores.t).sum(-1), 1.0 - beta ** Tq, rtol=1e-3)
+
+
 def test_importance_statistic_sum_is_the_prefix_call_and_bad_arguments_are_refused():
     rng = np.random.default_rng(3)
     N, H, Tq, P, D = 1, 2, 150, 20, 128
