@@ -5,7 +5,9 @@
 //
 // One CTA per SM works on two adjacent 128-row query tiles of one unit at a time (a work item),
 // each served by its own team of eight softmax warps; the key and value tiles stream once for
-// both, from the upper tile's diagonal down to tile 0. Per key tile and team:
+// both, from tile 0 up to the upper tile's diagonal (the lower tile's team stops one tile earlier
+// and normalises and stores its rows while the other team works on its diagonal tile). Per key
+// tile and team:
 //   S = Q K^T            tcgen05.mma, both operands K-major from TMA-staged shared memory, S in TMEM
 //   P = 2^(c*S - m)      the team reads S (one row per thread pair), writes P as bf16 over the
 //                        first half of S's own TMEM columns
@@ -187,8 +189,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     auto tmem_s = [&](uint32_t x) { return tmem_base + x * (uint32_t)kTileRows; };               // S (and P over its first half)
     auto tmem_o = [&](uint32_t x) { return tmem_base + 2u * kTileRows + x * (uint32_t)kTileRows; };
 
-    // item -> unit, upper query tile (team 0), its first (highest) key tile and number of key tiles.
-    // Team 1 takes the tile below (if there is one) and joins at the key tile that is its own first.
+    // item -> unit, upper query tile (team 0), its highest key tile and number of key tiles (streamed
+    // in ascending order). Team 1 takes the tile below (if there is one) and its own, smaller number.
     const int n_units = n_items / nps, head_items = (n_units - tail_units) * nps;
     auto decode_item = [&](int item, int &unit, int &a, int &first, int &count) {
         int k;
@@ -204,8 +206,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         first = geo.jmax(a);
         count = first + 1;
     };
-    // streamed index at which team 1 joins (count: never)
-    auto join_of = [&](int a, int first, int count) { return a >= 1 ? first - geo.jmax(a - 1) : count; };
+    // number of key tiles of team 1 (0: no tile below)
+    auto count1_of = [&](int a) { return a >= 1 ? geo.jmax(a - 1) + 1 : 0; };
 
     bool alive = true;
 
@@ -225,7 +227,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int next = grid_n + atomicAdd(next_item, 1);
                 for (int t = 0; t < count; ++t, ++tg) {
                     const uint32_t s = tg & 1u, ph = (tg >> 1) & 1u;
-                    const int row0 = (first - t) * kTileRows;
+                    const int row0 = t * kTileRows;
                     if (!mbar_wait(bar_k_empty(s), ph ^ 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                     mbar_expect_tx(bar_k_full(s), kTile);
 #pragma unroll
@@ -283,13 +285,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int4 d = sched_s[sl];
                 mbar_arrive(bar_sched_empty(sl));
                 if (d.x < 0) break;
-                const int count = d.w, join = join_of(d.y, d.z, d.w);
+                const int count = d.w, count1 = count1_of(d.y);
                 if (!mbar_wait(bar_q_full, it & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                // S of the first key tile (team 1 too if it joins at once)
+                // S of the first key tile for both teams
                 if (!mbar_wait(bar_k_full(tg & 1u), (tg >> 1) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                 tc_fence_after();
                 issue_s(0, tg & 1u);
-                if (join == 0) issue_s(1, tg & 1u);
+                if (count1 > 0) issue_s(1, tg & 1u);
                 umma_commit(bar_k_empty(tg & 1u));
                 if (count == 1) umma_commit(bar_q_empty);
                 for (int t = 0; t < count; ++t, ++tg) {
@@ -297,12 +299,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     const bool more = t + 1 < count;
                     const uint32_t s1 = (tg + 1u) & 1u, ph1 = ((tg + 1u) >> 1) & 1u;
                     for (uint32_t x = 0; x < 2; ++x) {
-                        if (x == 0 || t >= join) {
+                        const int cnt_x = x == 0 ? count : count1;
+                        if (t < cnt_x) {
                             // O += P V of team x for this key tile, then at once the team's S for the next one: both run
                             // while the other team does its softmax
                             if (!mbar_wait(bar_p_full(x), np[x] & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                             if (!mbar_wait(bar_v_full(s), ph, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
-                            const bool first_of_item = (x == 0) ? (t == 0) : (t == join);
+                            const bool first_of_item = t == 0;
                             // the team's previous output has been read out of TMEM before this item overwrites it
                             if (first_of_item && !mbar_wait(bar_o_free(x), (ni[x] + 1u) & 1u, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                             tc_fence_after();
@@ -312,9 +315,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                 umma_bf16_ts(tmem_o(x), tmem_s(x) + 8u * kk, umma_desc_mn(v0 + (uint32_t)kk * 2048u, kBoxBytes, 1024u),
                                              kIdescO, (!first_of_item || kk > 0) ? 1u : 0u);
                             ++np[x];
-                            if (!more) { umma_commit(bar_pv_done(x)); ++ni[x]; }
+                            if (t + 1 == cnt_x) { umma_commit(bar_pv_done(x)); ++ni[x]; }    // the team's last product of the item
                         }
-                        if (more && (x == 0 || t + 1 >= join)) {
+                        if (t + 1 < cnt_x) {
                             if (x == 0) {
                                 if (!mbar_wait(bar_k_full(s1), ph1, abort_flag, status, kWaitLimitNs, kPollBackoffNs)) { alive = false; break; }
                                 tc_fence_after();
@@ -353,13 +356,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_sched_empty(sl));
             if (d.x < 0) break;
-            const int unit = d.x, st = d.y - (int)x, first = d.z, count = d.w;
-            const int t0 = x == 0 ? 0 : join_of(d.y, d.z, d.w);           // first streamed index this team works on
-            if (t0 >= count) continue;                                    // no tile for this team in this item
+            const int unit = d.x, st = d.y - (int)x;
+            const int count = x == 0 ? d.w : count1_of(d.y);              // key tiles 0 .. count-1 for this team
+            if (count == 0) continue;                                     // no tile for this team in this item
             float m_ref = -INFINITY, l = 0.f;                 // running maximum (log2 domain) and this half's row sum
-            for (int t = t0; t < count; ++t, ++n) {
-                const int tile = first - t;
-                const int off = (st - tile) * kTileRows + geo.P;          // column col of the tile is visible iff col <= r + off
+            for (int t = 0; t < count; ++t, ++n) {
+                const int off = (st - t) * kTileRows + geo.P;             // column col of key tile t is visible iff col <= r + off
                 if (!mbar_wait(bar_s_full(x), n & 1u, abort_flag, status)) { alive = false; break; }
                 tc_fence_after();
                 float v[64];
