@@ -114,6 +114,12 @@ importance_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     }
+    // The kernel behind this one on the stream (pass 2 behind pass 1, the selection behind pass 2) may be
+    // scheduled as soon as CTAs of this one leave; it waits for this grid to finish before it reads anything.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Pass 2 is launched with programmatic stream serialization: its CTAs take the places pass-1 CTAs
+    // free and wait here, so the launch latency falls under pass 1's tail. (A no-op otherwise.)
+    if (PASS2) asm volatile("griddepcontrol.wait;" ::: "memory");
     // a CTA of this launch has already given up: leave at once instead of timing out again
     if (threadIdx.x == 0) *abort_flag = *reinterpret_cast<volatile int *>(status);
     __syncthreads();
@@ -498,13 +504,25 @@ cudaError_t launch_passes(const CUtensorMap &mq, const CUtensorMap &mk, int unit
     if (first_pass)
         importance_kernel<D, STAGES, kPass1><<<grid1, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)items1, tail1, c, lse2,
                                                                               lse_out, scores, status, status + 1);
+    cudaError_t e1 = cudaGetLastError();
+    if (e1 != cudaSuccess) return e1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int n2 = (int)items2;
+    int *counter2 = status + 2;
     if (take_max)
-        importance_kernel<D, STAGES, kPass2Max><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)items2, tail2, c, lse2,
-                                                                                 lse_out, scores, status, status + 2);
-    else
-        importance_kernel<D, STAGES, kPass2Sum><<<grid2, kThreads, smem, stream>>>(mq, mk, geo, fold, (int)items2, tail2, c, lse2,
-                                                                                 lse_out, scores, status, status + 2);
-    return cudaGetLastError();
+        return cudaLaunchKernelEx(&cfg, importance_kernel<D, STAGES, kPass2Max>, mq, mk, geo, fold, n2, tail2, c, lse2, lse_out,
+                                  scores, status, counter2);
+    return cudaLaunchKernelEx(&cfg, importance_kernel<D, STAGES, kPass2Sum>, mq, mk, geo, fold, n2, tail2, c, lse2, lse_out,
+                              scores, status, counter2);
 }
 
 }  // namespace

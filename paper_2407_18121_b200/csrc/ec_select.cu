@@ -84,6 +84,9 @@ select_kernel(const float *__restrict__ scores, int n_units, int T, int C, int p
     __shared__ uint32_t xa[2][kMaxWarpsPerUnit], xc[2][kMaxWarpsPerUnit];   // cross-warp exchange (G > 1), double-buffered
     extern __shared__ uint32_t planes_all[];                               // 32 x 32 words per warp
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // launched with programmatic stream serialization: the kernel in front (normally the importance
+    // kernel's column-sum pass) must have finished before the scores are read
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int unit = (G == 1) ? blockIdx.x * 4 + warp : blockIdx.x;
     if (G == 1 && unit >= n_units) return;                 // whole warp leaves; no barriers in this variant
     const int wu = (G == 1) ? 0 : warp;                    // this warp's index inside the unit
@@ -252,9 +255,17 @@ cudaError_t launch_select_t(const float *scores, int n_units, int T, int n_keep,
         cudaError_t e = cudaFuncSetAttribute(select_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
     }
-    select_kernel<G><<<grid, G == 1 ? 128 : 32 * G, smem, stream>>>(scores, n_units, T, n_keep, protect_ends, replicate,
-                                                                 anchor_pos, bucket_len);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(G == 1 ? 128 : 32 * G);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, select_kernel<G>, scores, n_units, T, n_keep, protect_ends, replicate, anchor_pos, bucket_len);
 }
 }  // namespace
 

@@ -3,6 +3,7 @@ workload shape and sequences the three calls. No arithmetic happens here.
 
     s = ElasticCacheSession(N, H, T, D, keep_ratio=0.5, offset=16, scale=1/sqrt(D))
     s.compress(Q, K, V)                  # importance -> select/merge; cache ready, len = budget
+    s.compress_with_attention(Q, K, V, out)   # the same, with the prompt's attention output as a by-product
     s.decode(q_all, k_all, v_all, out)   # [steps, N, H, D] each; fixed-point eviction every step
 
 `compress_host` / `decode_host` take pinned host tensors and include the host<->device
@@ -51,6 +52,17 @@ class ElasticCacheSession:
     def compress(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor) -> None:
         """Prompt call: importance, anchor selection and merge. Resets the cache to `n_keep` rows."""
         ec.ec_importance(Q, K, self.scores, None, self.scale, self.ws_imp)
+        ec.ec_select_merge(K, V, self.scores, self.n_keep, self.population, self.protect_ends,
+                           self.Kc, self.Vc, self.anchor_pos, None, self.ws_sel)
+        self.cache = ec.ec_cache_init(self.Kc, self.Vc, self.n_keep, max(self.n_keep, 2),
+                                      min(self.offset, max(self.n_keep, 2) - 1))
+
+    def compress_with_attention(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, out: torch.Tensor,
+                                lse: Optional[torch.Tensor] = None) -> None:
+        """compress() for callers that also want the prompt's attention output (the model's own forward
+        pass): `out` [N,H,T,D] and optionally `lse` [N,H,T] come from ec_prefill_attention, whose
+        normaliser also gives the importance by the column-sum pass alone. Same cache afterwards."""
+        ec.ec_prefill_attention(Q, K, V, out, lse, self.scores, self.scale, self.ws_imp)
         ec.ec_select_merge(K, V, self.scores, self.n_keep, self.population, self.protect_ends,
                            self.Kc, self.Vc, self.anchor_pos, None, self.ws_sel)
         self.cache = ec.ec_cache_init(self.Kc, self.Vc, self.n_keep, max(self.n_keep, 2),

@@ -147,3 +147,27 @@ def test_prefill_attention_long_context_units_full_length():
     # 8192-token units of the long-context configuration (64 key tiles per query tile at the end)
     w = wl.WORKLOADS["long8k"]
     _check_sampled_rows(w, [0, 1], [(0, 0), (1, 31)], [(0, 129), (4000, 4100), (8064, 8192)])
+
+
+def test_session_compress_with_attention_gives_the_same_cache():
+    # the prompt call through the attention kernel: the anchors and the merged cache are those of the
+    # two-pass call wherever the scores do not tie at the threshold (they agree to a few fp32 ulps)
+    from paper_2407_18121_b200.session import ElasticCacheSession
+    w = wl.WORKLOADS["tiny"]
+    Qb, Kb, Vb = wl.prompt(w)
+    N, H, T, D = Qb.shape
+    Q, K, V = dev_bf16(Qb), dev_bf16(Kb), dev_bf16(Vb)
+    a = ElasticCacheSession(N, H, T, D, w.keep_ratio, w.offset, w.scale)
+    b = ElasticCacheSession(N, H, T, D, w.keep_ratio, w.offset, w.scale)
+    a.compress(Q, K, V)
+    out = torch.empty_like(Q)
+    b.compress_with_attention(Q, K, V, out)
+    assert ec.ec_device_status(b.ws_imp) == ec.EC_OK
+    want_out, _ = orc.attention_prefix(Qb, Kb, Vb, w.scale)
+    assert_bf16_close(out, want_out, "attention output through the session")
+    torch.testing.assert_close(b.scores, a.scores, rtol=2e-4, atol=0)
+    same = (a.anchor_pos == b.anchor_pos).all(dim=-1)
+    assert same.float().mean().item() >= 0.75
+    assert torch.equal(a.Kc[same].view(torch.int16), b.Kc[same].view(torch.int16))
+    assert torch.equal(a.Vc[same].view(torch.int16), b.Vc[same].view(torch.int16))
+    assert b.cache.len == b.n_keep
