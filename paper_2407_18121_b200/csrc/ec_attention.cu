@@ -151,6 +151,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
     }
+    // the column-sum pass that may follow is launched with programmatic stream serialization: it may be
+    // scheduled as CTAs of this grid leave, and waits for the whole grid before it reads the normaliser
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) *abort_flag = *reinterpret_cast<volatile int *>(status);
     __syncthreads();
     if (*abort_flag) return;
