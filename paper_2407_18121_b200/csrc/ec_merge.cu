@@ -23,7 +23,7 @@ namespace {
 #define EC_MERGE_UNROLL 8
 #endif
 #ifndef EC_MERGE_MIN_CTAS
-#define EC_MERGE_MIN_CTAS 1
+#define EC_MERGE_MIN_CTAS 8      // 64 registers: eight CTAs per SM (68 registers and seven CTAs without the bound)
 #endif
 constexpr int kMergeThreads = EC_MERGE_THREADS;
 constexpr int kRowsPerCta = EC_MERGE_ROWS_PER_CTA;
