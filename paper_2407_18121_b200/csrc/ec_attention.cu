@@ -30,8 +30,6 @@
 // records a status word and leaves.
 #include "ec_tc.cuh"
 
-#include <type_traits>
-
 namespace ec {
 
 namespace {

@@ -129,6 +129,25 @@ def test_statistic_prefix_and_from_lse_reject_bad_arguments_on_the_host(L):
     assert h(p, p, p, p, 1, 1, 16, 32, 1.0, p, ws, None) == 2
 
 
+def test_prefill_attention_rejects_bad_arguments_on_the_host(L):
+    p = 0x10000
+    f = L.ec_prefill_attention
+    ws = 1 << 20
+    # (Q, K, V, out, lse, scores, N, H, Tq, P, D, scale, ws, ws_bytes, stream); nothing is launched on an error
+    assert f(None, p, p, p, None, None, 1, 1, 16, 0, 64, 1.0, p, ws, None) == 1
+    assert f(p, p, None, p, None, None, 1, 1, 16, 0, 64, 1.0, p, ws, None) == 1
+    assert f(p, p, p, None, None, None, 1, 1, 16, 0, 64, 1.0, p, ws, None) == 1
+    assert f(p, p, p, p, None, None, 1, 1, 16, 0, 48, 1.0, p, ws, None) == 2          # head dimension
+    assert f(p, p, p, p, None, None, 1, 1, 0, 0, 64, 1.0, p, ws, None) == 2           # no queries
+    assert f(p, p, p, p, None, None, 1, 1, 16, -1, 64, 1.0, p, ws, None) == 2         # negative prefix
+    assert f(p, p, p, p, None, None, 1, 1, 16, 0, 64, 0.0, p, ws, None) == 4          # scale
+    assert f(p, p, p + 8, p, None, None, 1, 1, 16, 0, 64, 1.0, p, ws, None) == 3      # V misaligned
+    assert f(p, p, p, p, p + 4, None, 1, 1, 16, 0, 64, 1.0, p, ws, None) == 3         # lse misaligned
+    assert f(p, p, p, p, None, None, 1, 1, 16, 0, 64, 1.0, None, 0, None) == 5
+    assert f(p, p, p, p, None, None, 1, 1, 16, 0, 64, 1.0, p, 64, None) == 5          # workspace too small
+    assert f(p, p, p, p, None, None, 1, 1, 16, 0, 64, 1.0, p + 16, ws, None) == 3     # workspace misaligned
+
+
 def test_cache_concat_rejects_bad_arguments_on_the_host(L):
     p = 0x10000
     c = ec.ec_cache()
