@@ -11,7 +11,7 @@
  * A "unit" is one (problem, head) pair; units are independent (OpenMP runs them in
  * parallel, which changes no result).
  *
- * Readings of the paper taken here (each is also listed in the design notes):
+ * Readings of the paper taken here:
  *  - Eq. 1: ordinary causal softmax, the denominator runs over keys m' <= m, so every
  *    row of A sums to one. An explicit `scale` multiplies the dot product.
  *  - Positions are 0-based, 0..T-1; Eq. 2's last bucket ends at T-1 and every bucket
