@@ -27,7 +27,10 @@ constexpr int kDecThreads = EC_DEC_THREADS;
 #define EC_DEC_TARGET (148 * 4)
 #endif
 constexpr int kMaxSplits = EC_DEC_TARGET;     // CTAs aimed at when there are fewer units than that; also the most splits a unit gets
-constexpr int kMinRowsPerSplit = 256;
+#ifndef EC_DEC_MIN_ROWS
+#define EC_DEC_MIN_ROWS 256
+#endif
+constexpr int kMinRowsPerSplit = EC_DEC_MIN_ROWS;
 constexpr int kBlk = 8;                       // rows per block of a lane group
 
 // The cache is written later in the same kernel, so no read-only (.nc) path here.
@@ -144,14 +147,17 @@ __device__ __forceinline__ void process_block(GroupState &st, const float2 (&q2)
 // splits  > 1: every CTA writes (acc[D], max, sum) of its rows to `partials` and counts itself in
 // `counters[unit]`; the CTA that arrives last (nobody waits for anybody) merges the unit's partials,
 // writes out, stores the new row and puts the counter back to zero for the next launch.
-template <int LPR>
-__global__ void __launch_bounds__(kDecThreads, EC_DEC_MIN_CTAS)
+// THREADS = 64 is the shape for launches that fill the GPU. When a launch has too few CTAs for that (a
+// single layer's units), wider CTAs give a unit more lane groups, so that a group walks one or two blocks
+// of rows instead of four or five one after the other: the step is then a shorter chain of memory round trips.
+template <int LPR, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == kDecThreads ? EC_DEC_MIN_CTAS : 1)
 decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
               uint4 *Kc, uint4 *Vc, int cap, int len, int write_slot, int defer_from, float scale_log2e,
               __nv_bfloat16 *__restrict__ out, float *partials, int *counters, int splits, int release_early)
 {
     constexpr int D = LPR * 8;
-    constexpr int G = kDecThreads / LPR;
+    constexpr int G = THREADS / LPR;
     __shared__ float sm_acc[G][D];
     __shared__ float sm_m[G], sm_l[G];
     __shared__ int sm_last;
@@ -246,7 +252,7 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
     }
     __syncthreads();   // also orders every cache read of this CTA before the slot write below
 
-    for (int d = threadIdx.x; d < D; d += kDecThreads) {
+    for (int d = threadIdx.x; d < D; d += THREADS) {
         float M = -INFINITY;
 #pragma unroll
         for (int gg = 0; gg < G; ++gg) M = fmaxf(M, sm_m[gg]);
@@ -279,7 +285,7 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
             if (threadIdx.x == 0) counters[unit] = 0;
             // the splits' (max, sum) pairs first, all loads in flight at once, then their weights
             const float *p = partials + (size_t)unit * splits * (D + 2);
-            for (int sp = threadIdx.x; sp < splits; sp += kDecThreads) {
+            for (int sp = threadIdx.x; sp < splits; sp += THREADS) {
                 sm_pm[sp] = __ldcg(p + (size_t)sp * (D + 2) + D);
                 sm_pl[sp] = __ldcg(p + (size_t)sp * (D + 2) + D + 1);
             }
@@ -292,7 +298,7 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
                 L = fmaf(sm_pl[sp], (ms == -INFINITY) ? 0.f : fast_exp2(ms - M), L);
             }
             const float inv_l = 1.f / L;
-            for (int d = threadIdx.x; d < D; d += kDecThreads) {
+            for (int d = threadIdx.x; d < D; d += THREADS) {
                 float A = 0.f;
 #pragma unroll 4
                 for (int sp = 0; sp < splits; ++sp) {
@@ -304,8 +310,8 @@ decode_kernel(const uint4 *__restrict__ q, const uint4 *__restrict__ k_new, cons
         }
     }
     // the new row takes the freed slot once every CTA of the unit has read its rows
-    if (finish && threadIdx.x >= kDecThreads - 2 * LPR) {
-        const int i = threadIdx.x - (kDecThreads - 2 * LPR);
+    if (finish && threadIdx.x >= THREADS - 2 * LPR) {
+        const int i = threadIdx.x - (THREADS - 2 * LPR);
         if (i < LPR) Kcu[(size_t)write_slot * LPR + i] = knu[i];
         else         Vcu[(size_t)write_slot * LPR + (i - LPR)] = vnu[i - LPR];
     }
@@ -347,6 +353,19 @@ cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, unsigned 
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+int sm_count_cached()
+{
+    static int n = 0;
+    if (n < 1) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            return 148;
+    }
+    return n;
+}
+
 template <int LPR>
 cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc, int units,
                             int cap, int len, int write_slot, int defer_from, float sl2, void *out, float *partials,
@@ -356,9 +375,17 @@ cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new,
 #define EC_DEC_EARLY_MIN_MB 24
 #endif
     const int release_early = (double)units * len * LPR * 32.0 >= EC_DEC_EARLY_MIN_MB * 1.0e6;   // K and V bytes of a step
-    return launch_overlapped(decode_kernel<LPR>, (unsigned)(units * splits), (unsigned)kDecThreads, stream,
-                             (const uint4 *)q, (const uint4 *)k_new, (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap, len,
-                             write_slot, defer_from, sl2, (__nv_bfloat16 *)out, partials, counters, splits, release_early);
+    // the widest CTA with which the whole launch is still resident at once (about 512 threads per SM at this
+    // kernel's register count)
+    const long long ctas = (long long)units * splits, resident_threads = 512LL * sm_count_cached();
+    auto go = [&](auto kernel, unsigned threads) {
+        return launch_overlapped(kernel, (unsigned)ctas, threads, stream, (const uint4 *)q, (const uint4 *)k_new,
+                                 (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap, len, write_slot, defer_from, sl2,
+                                 (__nv_bfloat16 *)out, partials, counters, splits, release_early);
+    };
+    if (ctas * 256 <= resident_threads) return go(decode_kernel<LPR, 256>, 256u);
+    if (ctas * 128 <= resident_threads) return go(decode_kernel<LPR, 128>, 128u);
+    return go(decode_kernel<LPR, kDecThreads>, (unsigned)kDecThreads);
 }
 
 cudaError_t launch_decode(const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
