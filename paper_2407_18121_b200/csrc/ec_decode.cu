@@ -377,7 +377,10 @@ cudaError_t launch_decode_t(const void *q, const void *k_new, const void *v_new,
     const int release_early = (double)units * len * LPR * 32.0 >= EC_DEC_EARLY_MIN_MB * 1.0e6;   // K and V bytes of a step
     // the widest CTA with which the whole launch is still resident at once (about 512 threads per SM at this
     // kernel's register count)
-    const long long ctas = (long long)units * splits, resident_threads = 512LL * sm_count_cached();
+    #ifndef EC_DEC_WIDE_X2
+#define EC_DEC_WIDE_X2 2      // twice the factor by which a wide launch may exceed what is resident at once
+#endif
+    const long long ctas = (long long)units * splits, resident_threads = 512LL * sm_count_cached() * EC_DEC_WIDE_X2 / 2;
     auto go = [&](auto kernel, unsigned threads) {
         return launch_overlapped(kernel, (unsigned)ctas, threads, stream, (const uint4 *)q, (const uint4 *)k_new,
                                  (const uint4 *)v_new, (uint4 *)Kc, (uint4 *)Vc, cap, len, write_slot, defer_from, sl2,
